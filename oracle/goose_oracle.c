@@ -1,0 +1,260 @@
+/*
+ * CPU oracle for the Goose tree-verification step.  TEST INFRASTRUCTURE ONLY.
+ *
+ * Plain, slow, fp64, written from the paper's definitions; it shares no code, header,
+ * table or helper with the CUDA library and must never be called from the product path
+ * (only the tests, the smoke check and the benchmark's CPU-baseline leg use it).
+ *
+ * Every function below is the plain definition of what the step computes:
+ *   - tree attention:  the "tree attention mask ... lets each node attend only to its
+ *     root-to-node ancestors" (Sec. 4, Stage 1; Algorithm 1 "Ensure"; Algorithm 3 step 1),
+ *     i.e. softmax(scale * q.K^T + mask) V with mask = prefix + ancestors (self included).
+ *   - node top-k:      per-node greedy argmax (Algorithm 3 step 2) and the batched top-K
+ *     harvested from every row of the forward's logits (App. "Aggressive logit harvesting").
+ *   - accept:          UnifiedGreedyWalk (Algorithm 3), literal pointer walk.
+ *   - kv compaction:   the paper never describes it; the reading used here is "keep the
+ *     accepted nodes' K/V rows, in path order, directly after the prefix".
+ *
+ * bf16 inputs arrive as uint16 bit patterns; bf16 -> double is exact.
+ * No blocking, no fusion, no reordering: one output element at a time.
+ * All functions are pinned by tests that do not depend on this file's own formulas.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static double bf16_to_f64(uint16_t b) {
+    uint32_t u = ((uint32_t)b) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ------------------------------------------------------------------ ancestors
+ * A(0) = {0};  A(i) = A(parent[i]) U {i}   (root-to-node path, node included).
+ * vis[j] = 1 iff j in A(i).  Returns 0, or -1 if parent[] is not a rooted tree in
+ * topological order (parent[0] = -1, 0 <= parent[i] < i). */
+static int ancestors_of(const int32_t* parent, int B, int i, unsigned char* vis) {
+    memset(vis, 0, (size_t)B);
+    int v = i;
+    int steps = 0;
+    while (v != -1) {
+        if (v < 0 || v >= B || steps > B) return -1;
+        vis[v] = 1;
+        int p = parent[v];
+        if (v == 0) {
+            if (p != -1) return -1;
+        } else if (p < 0 || p >= v) {
+            return -1;
+        }
+        v = p;
+        ++steps;
+    }
+    return vis[0] ? 0 : -1;
+}
+
+int oracle_check_parent(const int32_t* parent, int B) {
+    if (B < 1 || parent[0] != -1) return -1;
+    for (int i = 1; i < B; ++i)
+        if (parent[i] < 0 || parent[i] >= i) return -1;
+    return 0;
+}
+
+/* ------------------------------------------------------------------ tree attention, one row
+ * Node i of sequence s, head h.  Visible keys: prefix rows 0..ctx-1 and tree rows ctx+j, j in A(i).
+ *   s_j = scale * sum_d q[d] K[j][d];  p_j = exp(s_j - max) / sum exp(s - max);  out = sum_j p_j V[j].
+ * K/V layout: [row][H][D], sequence s owns rows row_off[s] .. row_off[s]+ctx+B-1. */
+static int attn_row(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, int64_t row0, int ctx,
+                    const int32_t* parent, int B, int H, int D, double scale, int i, int h,
+                    const uint16_t* qrow /* q[s][i][h][:] */, double* out /* [D] */, double* lse) {
+    (void)q;
+    int n = ctx + B;
+    unsigned char* vis = (unsigned char*)malloc((size_t)B);
+    double* sc = (double*)malloc(sizeof(double) * (size_t)n);
+    if (!vis || !sc) { free(vis); free(sc); return -2; }
+    if (ancestors_of(parent, B, i, vis) != 0) { free(vis); free(sc); return -1; }
+
+    double mx = -INFINITY;
+    for (int j = 0; j < n; ++j) {
+        int visible = (j < ctx) ? 1 : vis[j - ctx];
+        if (!visible) { sc[j] = -INFINITY; continue; }
+        const uint16_t* krow = kc + ((size_t)(row0 + j) * H + h) * D;
+        double acc = 0.0;
+        for (int d = 0; d < D; ++d) acc += bf16_to_f64(qrow[d]) * bf16_to_f64(krow[d]);
+        sc[j] = scale * acc;
+        if (sc[j] > mx) mx = sc[j];
+    }
+    double denom = 0.0;
+    for (int j = 0; j < n; ++j)
+        if (sc[j] != -INFINITY) denom += exp(sc[j] - mx);
+    for (int d = 0; d < D; ++d) out[d] = 0.0;
+    for (int j = 0; j < n; ++j) {
+        if (sc[j] == -INFINITY) continue;
+        double p = exp(sc[j] - mx) / denom;
+        const uint16_t* vrow = vc + ((size_t)(row0 + j) * H + h) * D;
+        for (int d = 0; d < D; ++d) out[d] += p * bf16_to_f64(vrow[d]);
+    }
+    if (lse) *lse = mx + log(denom);
+    free(vis);
+    free(sc);
+    return 0;
+}
+
+/* Full output: out fp64 [S][B][H][D], lse fp64 [S][B][H] (may be NULL). Returns 0 or <0. */
+int oracle_tree_attn(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, const int64_t* row_off,
+                     const int32_t* ctx_len, const int32_t* parent, int S, int B, int H, int D,
+                     double scale, double* out, double* lse) {
+    int rc = 0;
+    long total = (long)S * B * H;
+#pragma omp parallel for schedule(dynamic, 4)
+    for (long t = 0; t < total; ++t) {
+        int h = (int)(t % H);
+        int i = (int)((t / H) % B);
+        int s = (int)(t / ((long)H * B));
+        const uint16_t* qrow = q + (((size_t)s * B + i) * H + h) * D;
+        int r = attn_row(q, kc, vc, row_off[s], ctx_len[s], parent + (size_t)s * B, B, H, D, scale, i, h, qrow,
+                         out + (size_t)t * D, lse ? lse + t : NULL);
+        if (r != 0) {
+#pragma omp critical
+            rc = r;
+        }
+    }
+    return rc;
+}
+
+/* Sampled rows: for each sample n the row (s,i,h) = (ss[n], si[n], sh[n]); out [n][D], lse [n]. */
+int oracle_tree_attn_rows(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, const int64_t* row_off,
+                          const int32_t* ctx_len, const int32_t* parent, int S, int B, int H, int D,
+                          double scale, int n_samples, const int32_t* ss, const int32_t* si,
+                          const int32_t* sh, double* out, double* lse) {
+    int rc = 0;
+    (void)S;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int n = 0; n < n_samples; ++n) {
+        int s = ss[n], i = si[n], h = sh[n];
+        const uint16_t* qrow = q + (((size_t)s * B + i) * H + h) * D;
+        int r = attn_row(q, kc, vc, row_off[s], ctx_len[s], parent + (size_t)s * B, B, H, D, scale, i, h, qrow,
+                         out + (size_t)n * D, lse ? lse + n : NULL);
+        if (r != 0) {
+#pragma omp critical
+            rc = r;
+        }
+    }
+    return rc;
+}
+
+/* ------------------------------------------------------------------ per-node argmax + top-k
+ * Order the indices of a row by (value descending, index ascending), values compared as real
+ * numbers (so -0.0 == +0.0); the first k are the top-k, the first one is the greedy argmax. */
+typedef struct { double v; int32_t idx; } vi_t;
+
+static int cmp_vi(const void* a, const void* b) {
+    const vi_t* x = (const vi_t*)a;
+    const vi_t* y = (const vi_t*)b;
+    if (x->v > y->v) return -1;
+    if (x->v < y->v) return 1;
+    return (x->idx > y->idx) - (x->idx < y->idx);
+}
+
+int oracle_node_topk(const uint16_t* logits, int rows, int V, int64_t ldl, int k,
+                     int32_t* argmax, int32_t* topk_ids, double* topk_vals) {
+    if (k < 1 || k > V) return -1;
+    int rc = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int r = 0; r < rows; ++r) {
+        vi_t* a = (vi_t*)malloc(sizeof(vi_t) * (size_t)V);
+        if (!a) {
+#pragma omp critical
+            rc = -2;
+            continue;
+        }
+        for (int j = 0; j < V; ++j) {
+            a[j].v = bf16_to_f64(logits[(size_t)r * ldl + j]);
+            a[j].idx = j;
+        }
+        qsort(a, (size_t)V, sizeof(vi_t), cmp_vi);   /* full sort; (value, index) is a total order */
+        argmax[r] = a[0].idx;
+        for (int j = 0; j < k; ++j) {
+            topk_ids[(size_t)r * k + j] = a[j].idx;
+            if (topk_vals) topk_vals[(size_t)r * k + j] = a[j].v;
+        }
+        free(a);
+    }
+    return rc;
+}
+
+/* ------------------------------------------------------------------ UnifiedGreedyWalk (Algorithm 3)
+ * v <- root; while v has children: if a spine-tagged child's token equals argmax[v] take it;
+ * else if a branch-tagged child's token equals argmax[v] take it; else stop.  bonus = argmax[v].
+ * tag == NULL: no source tags; the matching child with the lowest index is taken (with distinct
+ * sibling tokens at most one child can match, so the priority never changes the path).
+ * path [S][B]: path[0] = 0, then the accepted nodes, then -1.  accept_len excludes the root. */
+int oracle_accept(const int32_t* draft_tok, const int32_t* parent, const int32_t* argmax,
+                  const unsigned char* tag /* [S][B], 1 = spine child; or NULL */,
+                  int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus) {
+    for (int s = 0; s < S; ++s) {
+        const int32_t* par = parent + (size_t)s * B;
+        const int32_t* tok = draft_tok + (size_t)s * B;
+        const int32_t* am = argmax + (size_t)s * B;
+        int32_t* p = path + (size_t)s * B;
+        if (oracle_check_parent(par, B) != 0) return -1;
+        for (int j = 0; j < B; ++j) p[j] = -1;
+        int v = 0, len = 0;
+        p[0] = 0;
+        for (;;) {
+            int next = -1;
+            if (tag) {
+                for (int c = v + 1; c < B && next < 0; ++c)      /* priority 1: spine child */
+                    if (par[c] == v && tag[(size_t)s * B + c] && tok[c] == am[v]) next = c;
+                for (int c = v + 1; c < B && next < 0; ++c)      /* priority 2: branch children */
+                    if (par[c] == v && !tag[(size_t)s * B + c] && tok[c] == am[v]) next = c;
+            } else {
+                for (int c = v + 1; c < B && next < 0; ++c)
+                    if (par[c] == v && tok[c] == am[v]) next = c;
+            }
+            if (next < 0) break;
+            ++len;
+            p[len] = next;
+            v = next;
+        }
+        accept_len[s] = len;
+        bonus[s] = am[v];
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------ KV compaction (out of place)
+ * k_out/v_out start as copies of the caches; row ctx+j <- row ctx+path[j] of the ORIGINAL cache,
+ * j = 0..accept_len.  new_ctx = ctx + 1 + accept_len.  Rows >= new_ctx are left as they were. */
+int oracle_kv_compact(const uint16_t* kc, const uint16_t* vc, const int64_t* row_off, const int32_t* ctx_len,
+                      const int32_t* path, const int32_t* accept_len, int S, int B, int H, int D,
+                      uint16_t* k_out, uint16_t* v_out, int32_t* new_ctx) {
+    size_t row_elems = (size_t)H * D;
+    for (int s = 0; s < S; ++s) {
+        int L = accept_len[s];
+        if (L < 0 || L >= B) return -1;
+        for (int j = 0; j <= L; ++j) {
+            int src = path[(size_t)s * B + j];
+            if (src < 0 || src >= B) return -1;
+            size_t dst_row = (size_t)(row_off[s] + ctx_len[s] + j);
+            size_t src_row = (size_t)(row_off[s] + ctx_len[s] + src);
+            memcpy(k_out + dst_row * row_elems, kc + src_row * row_elems, row_elems * sizeof(uint16_t));
+            memcpy(v_out + dst_row * row_elems, vc + src_row * row_elems, row_elems * sizeof(uint16_t));
+        }
+        new_ctx[s] = ctx_len[s] + 1 + L;
+    }
+    return 0;
+}

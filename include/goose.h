@@ -1,0 +1,164 @@
+/*
+ * goose.h -- C ABI of the B200 (sm_100a) tree-verification step of Goose.
+ *
+ * One verification step scores a spine tree of B draft tokens in a single pass
+ * (Sec. 4, Stages 2-3; Algorithm 3):
+ *   goose_tree_attn   tree-masked attention of the B draft queries over the prefix KV cache
+ *                     plus each node's in-tree ancestors,
+ *   goose_node_topk   per-node greedy argmax and top-k of the vocabulary logits,
+ *   goose_accept      the greedy longest-accepted-path walk,
+ *   goose_kv_compact  in-place compaction of the accepted nodes' K/V rows.
+ *
+ * Conventions (all entry points)
+ *   - Every data pointer is a DEVICE pointer owned by the caller unless the argument is
+ *     documented as "host".  The library owns only the workspace inside goose_ctx.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default
+ *     stream), never synchronise the host, and return as soon as the work is enqueued.
+ *     goose_verify_step_host and goose_last_status are the exceptions: they synchronise.
+ *   - bf16 tensors are passed as void*; "bf16 [a][b]" means row-major, last index fastest.
+ *   - Return value: GOOSE_OK, or a negative code.  Argument errors are detected on the host
+ *     before anything is enqueued.  Data-dependent errors (an invalid parent[] array) are
+ *     detected on the device: the affected sequence gets zero-filled / neutral outputs and a
+ *     non-zero status word (goose_last_status); a kernel never traps and never spins without
+ *     a bound.
+ *   - A goose_ctx must not be used from two streams at once (its workspace is shared).
+ *
+ * Tree layout (Algorithm 1): node 0 is the anchor/root and counts towards B;
+ * parent[0] = -1 and 0 <= parent[i] < i (topological order).  B <= GOOSE_MAX_B.
+ *
+ * KV cache layout: bf16 [kv_rows][H][D], token-major.  Sequence s owns rows
+ * row_off[s] .. row_off[s] + ctx_len[s] + B - 1: first its ctx_len[s] prefix tokens, then the
+ * K/V of tree node i at row row_off[s] + ctx_len[s] + i (written by the caller before the call).
+ */
+#ifndef GOOSE_H_
+#define GOOSE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GOOSE_OK        0
+#define GOOSE_EINVAL   (-1)   /* bad argument (null / misaligned pointer, size out of range)        */
+#define GOOSE_ENOMEM   (-2)   /* workspace allocation failed                                       */
+#define GOOSE_ECUDA    (-3)   /* a CUDA runtime / driver call failed; see goose_strerror           */
+#define GOOSE_ETIMEOUT (-4)   /* a bounded device-side wait gave up (reported by goose_last_status) */
+
+#define GOOSE_MAX_B     128   /* tree nodes per sequence (one 128-bit ancestor mask per node)      */
+#define GOOSE_MAX_K      16   /* top-k width                                                       */
+#define GOOSE_HEAD_DIM  128   /* the only supported head dimension                                 */
+#define GOOSE_MAX_V  262144   /* vocabulary size limit of goose_node_topk                          */
+
+/* per-sequence status bits (goose_last_status) */
+#define GOOSE_ST_BAD_PARENT   1   /* parent[] is not a rooted tree in topological order */
+#define GOOSE_ST_BAD_PATH     2   /* path[] / accept_len[] handed to goose_kv_compact is invalid */
+#define GOOSE_ST_TIMEOUT      4   /* a device-side wait ran out of polls */
+
+/* attention kernel selection (goose_set_attn_impl) */
+#define GOOSE_ATTN_AUTO  0
+#define GOOSE_ATTN_MMA   1    /* warp-level mma.sync flash-decode kernel (any B <= 128)            */
+#define GOOSE_ATTN_UMMA  2    /* tcgen05 + TMEM + TMA persistent kernel                            */
+
+typedef struct goose_ctx goose_ctx;
+
+/* Create a context on CUDA device `device`.  Allocates the workspace (split-KV partials,
+ * arrival counters, per-sequence status) for up to max_S sequences of up to max_B <= 128 nodes
+ * and max_H heads; head_dim must be 128.  *out is NULL on failure.                              */
+int goose_create(goose_ctx** out, int device, int max_S, int max_B, int max_H, int head_dim);
+
+/* Free the workspace.  The caller must have synchronised every stream that used the context.   */
+int goose_destroy(goose_ctx* ctx);
+
+/* Static description of a return code; for GOOSE_ECUDA the text of the last CUDA error seen
+ * by this thread is appended.  The pointer stays valid until the next call from this thread.   */
+const char* goose_strerror(int rc);
+
+/* Choose the attention kernel (GOOSE_ATTN_*).  AUTO picks per call from B and the problem size. */
+int goose_set_attn_impl(goose_ctx* ctx, int impl);
+
+/* Tree attention (Sec. 4 Stage 1 "tree attention mask"; Algorithm 3 step 1).
+ * For sequence s, head h, node i:  out[s][i][h][:] = softmax_j(scale * q[s][i][h] . K[j][h]) V[j][h]
+ * over the visible keys j = prefix rows 0..ctx_len[s]-1 and tree rows ctx_len[s]+a for every
+ * ancestor a of i, i included.  bf16 inputs, fp32 accumulation, bf16 output (round to nearest even).
+ *   q        bf16 [S][B][H][D]                       16-byte aligned
+ *   k_cache, v_cache  bf16 [kv_rows][H][D]           16-byte aligned; kv_rows = rows allocated
+ *   row_off  int64 [S], ctx_len int32 [S], parent int32 [S][B]   (device arrays)
+ *   out      bf16 [S][B][H][D]; lse fp32 [S][B][H] = log-sum-exp of the scaled scores, or NULL
+ * Rows row_off[s]+ctx_len[s]+B .. are never read as values (their contents may be anything).
+ * ctx_len[s] = 0 is legal.  S <= max_S, B <= max_B, H <= max_H, D == 128.                       */
+int goose_tree_attn(goose_ctx* ctx, const void* q, const void* k_cache, const void* v_cache, int64_t kv_rows,
+                    const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
+                    int S, int B, int H, int D, float scale, void* out, float* lse, void* stream);
+
+/* Per-node argmax and top-k (Algorithm 3 step 2; App. C.1 "aggressive logit harvesting": every
+ * row of the forward's logits is harvested, rejected branches included).
+ * For each of `rows` rows: the ids of the k largest of the first V values, ordered by
+ * (value descending, index ascending); -0.0 equals +0.0; argmax[r] = topk_ids[r][0].
+ *   logits bf16 [rows][ldl]  16-byte aligned, ldl % 8 == 0, ldl >= V, finite values
+ *   1 <= k <= min(V, GOOSE_MAX_K); V <= GOOSE_MAX_V
+ *   argmax int32 [rows]; topk_ids int32 [rows][k]; topk_vals fp32 [rows][k] (exact values) or NULL */
+int goose_node_topk(goose_ctx* ctx, const void* logits, int rows, int V, int64_t ldl, int k,
+                    int32_t* argmax, int32_t* topk_ids, float* topk_vals, void* stream);
+
+/* Greedy acceptance walk (Algorithm 3, UnifiedGreedyWalk).  From node 0, repeatedly move to the
+ * child c of the current node v with draft_tok[c] == argmax[v]; stop when no child matches.
+ * If sibling tokens are not distinct the matching child with the lowest index is taken.
+ *   draft_tok, parent, argmax  int32 [S][B]
+ *   path int32 [S][B]: path[s][0] = 0, then the accepted nodes in order, then -1
+ *   accept_len int32 [S]: accepted draft nodes, root excluded; bonus int32 [S] = argmax at the last
+ *   accepted node.  An invalid parent[] gives accept_len 0, path {0,-1,..}, bonus -1 and status.  */
+int goose_accept(goose_ctx* ctx, const int32_t* draft_tok, const int32_t* parent, const int32_t* argmax,
+                 int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus, void* stream);
+
+/* KV compaction.  The paper does not describe cache handling after acceptance; this call keeps
+ * the accepted nodes' rows in path order directly after the prefix, in place:
+ * row ctx_len[s]+j <- row ctx_len[s]+path[s][j] for j = 0..accept_len[s], for K and V;
+ * new_ctx_len[s] = ctx_len[s] + 1 + accept_len[s].  Rows >= new_ctx_len[s] are unspecified after
+ * the call.  path must be increasing (as goose_accept produces it).                              */
+int goose_kv_compact(goose_ctx* ctx, void* k_cache, void* v_cache, int64_t kv_rows,
+                     const int64_t* row_off, const int32_t* ctx_len, const int32_t* path,
+                     const int32_t* accept_len, int S, int B, int H, int D,
+                     int32_t* new_ctx_len, void* stream);
+
+/* The whole step on one stream, in data-flow order: tree attention, node top-k (rows = S*B),
+ * acceptance walk, KV compaction.  Arguments as in the four calls above.                         */
+int goose_verify_step(goose_ctx* ctx, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
+                      const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
+                      const int32_t* draft_tok, const void* logits, int64_t ldl,
+                      int S, int B, int H, int D, int V, int k, float scale,
+                      void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
+                      int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
+                      void* stream);
+
+/* Host-buffer variant of the whole step (the end-to-end call).  The prefix KV cache stays on the
+ * device (k_cache / v_cache are device pointers, state carried from step to step); everything a
+ * step consumes or produces is in HOST memory (pinned memory makes the copies asynchronous):
+ *   in : h_q bf16 [S][B][H][D]; h_k_new, h_v_new bf16 [S][B][H][D] = the tree nodes' K/V rows,
+ *        copied to rows row_off[s]+ctx_len[s]+i; h_row_off int64 [S]; h_ctx_len int32 [S];
+ *        h_parent, h_draft_tok int32 [S][B]; h_logits bf16 [S*B][V] (dense, ldl = V)
+ *   out: h_out bf16 [S][B][H][D]; h_argmax [S*B]; h_topk_ids [S*B][k]; h_topk_vals [S*B][k] or NULL;
+ *        h_path [S][B]; h_accept_len, h_bonus, h_new_ctx_len [S]
+ * Copies in, runs goose_verify_step, copies out, and synchronises `stream` before returning.
+ * Device staging buffers are allocated inside the context on first use and grow on demand.      */
+int goose_verify_step_host(goose_ctx* ctx, void* k_cache, void* v_cache, int64_t kv_rows,
+                           const void* h_q, const void* h_k_new, const void* h_v_new,
+                           const int64_t* h_row_off, const int32_t* h_ctx_len,
+                           const int32_t* h_parent, const int32_t* h_draft_tok, const void* h_logits,
+                           int S, int B, int H, int D, int V, int k, float scale,
+                           void* h_out, int32_t* h_argmax, int32_t* h_topk_ids, float* h_topk_vals,
+                           int32_t* h_path, int32_t* h_accept_len, int32_t* h_bonus,
+                           int32_t* h_new_ctx_len, void* stream);
+
+/* Synchronise the device, copy the per-sequence status words (GOOSE_ST_* bits, OR-ed over all
+ * calls since the last query) into host_status[0..S) (a HOST array) and clear them.
+ * Returns GOOSE_ETIMEOUT if any word has GOOSE_ST_TIMEOUT set.  For tests and debugging.         */
+int goose_last_status(goose_ctx* ctx, int32_t* host_status, int S);
+
+/* Number of kernels this library has launched through `ctx` since it was created.              */
+int64_t goose_launch_count(goose_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GOOSE_H_ */

@@ -1,0 +1,308 @@
+// C ABI of libgoose: context management, argument validation, and the entry points declared in goose.h.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "goose_internal.cuh"
+
+namespace {
+
+thread_local char g_errbuf[512];
+thread_local cudaError_t g_last_cuda = cudaSuccess;
+
+int cuda_fail(cudaError_t e) {
+    g_last_cuda = e;
+    return GOOSE_ECUDA;
+}
+#define GOOSE_CUDA(call)                         \
+    do {                                         \
+        cudaError_t e__ = (call);                \
+        if (e__ != cudaSuccess) return cuda_fail(e__); \
+    } while (0)
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_shape(const goose_ctx* c, int S, int B, int H, int D) {
+    if (!c) return GOOSE_EINVAL;
+    if (S < 0 || S > c->max_S) return GOOSE_EINVAL;
+    if (B < 1 || B > c->max_B || B > GOOSE_MAX_B) return GOOSE_EINVAL;
+    if (H < 1 || H > c->max_H) return GOOSE_EINVAL;
+    if (D != GOOSE_HEAD_DIM) return GOOSE_EINVAL;
+    return GOOSE_OK;
+}
+
+constexpr int kTopkChunkElems = 8192;
+constexpr int kTopkMaxChunks = GOOSE_MAX_V / kTopkChunkElems;   // 32
+
+}  // namespace
+
+extern "C" {
+
+const char* goose_strerror(int rc) {
+    const char* base;
+    switch (rc) {
+        case GOOSE_OK: base = "ok"; break;
+        case GOOSE_EINVAL: base = "invalid argument"; break;
+        case GOOSE_ENOMEM: base = "out of memory"; break;
+        case GOOSE_ECUDA: base = "CUDA error"; break;
+        case GOOSE_ETIMEOUT: base = "device-side wait timed out"; break;
+        default: base = "unknown error"; break;
+    }
+    if (rc == GOOSE_ECUDA)
+        snprintf(g_errbuf, sizeof g_errbuf, "%s: %s", base, cudaGetErrorString(g_last_cuda));
+    else
+        snprintf(g_errbuf, sizeof g_errbuf, "%s", base);
+    return g_errbuf;
+}
+
+int goose_create(goose_ctx** out, int device, int max_S, int max_B, int max_H, int head_dim) {
+    if (!out) return GOOSE_EINVAL;
+    *out = nullptr;
+    if (max_S < 1 || max_B < 1 || max_B > GOOSE_MAX_B || max_H < 1 || head_dim != GOOSE_HEAD_DIM) return GOOSE_EINVAL;
+    GOOSE_CUDA(cudaSetDevice(device));
+    goose_ctx* c = new (std::nothrow) goose_ctx();
+    if (!c) return GOOSE_ENOMEM;
+    memset(c, 0, sizeof *c);
+    c->device = device;
+    c->max_S = max_S; c->max_B = max_B; c->max_H = max_H;
+    c->attn_impl = GOOSE_ATTN_AUTO;
+    cudaDeviceProp prop;
+    cudaError_t e = cudaGetDeviceProperties(&prop, device);
+    if (e != cudaSuccess) { delete c; return cuda_fail(e); }
+    c->num_sms = prop.multiProcessorCount;
+
+    // attention partial slots: two per CTA of the persistent kernel, or heads x splits of the split kernel
+    long long heads = (long long)max_S * max_H;
+    long long slots = 2LL * c->num_sms + 2;
+    if (slots < heads) slots = heads;           // at least one slot per head
+    if (slots < 4LL * c->num_sms) slots = 4LL * c->num_sms;
+    c->n_slots = (int)slots;
+    c->topk_rows_cap = max_S * max_B;
+    c->topk_cand_cap = (int64_t)c->topk_rows_cap * kTopkMaxChunks * GOOSE_MAX_K;
+
+    bool ok = true;
+    ok = ok && cudaMalloc(&c->partials, sizeof(float) * (size_t)c->n_slots * goose::kPartialFloats) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->head_counters, sizeof(int32_t) * (size_t)heads) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->topk_cand, sizeof(unsigned long long) * (size_t)c->topk_cand_cap) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->row_counters, sizeof(int32_t) * (size_t)c->topk_rows_cap) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->status, sizeof(int32_t) * (size_t)max_S) == cudaSuccess;
+    if (ok) {
+        ok = ok && cudaMemset(c->head_counters, 0, sizeof(int32_t) * (size_t)heads) == cudaSuccess;
+        ok = ok && cudaMemset(c->row_counters, 0, sizeof(int32_t) * (size_t)c->topk_rows_cap) == cudaSuccess;
+        ok = ok && cudaMemset(c->status, 0, sizeof(int32_t) * (size_t)max_S) == cudaSuccess;
+    }
+    if (ok) {
+        cudaDriverEntryPointQueryResult qres;
+        void* fn = nullptr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            c->encode_tiled = fn;
+        ok = goose::init_kernels(c) == cudaSuccess;
+    }
+    if (!ok) {
+        cudaGetLastError();
+        goose_destroy(c);
+        return GOOSE_ENOMEM;
+    }
+    *out = c;
+    return GOOSE_OK;
+}
+
+int goose_destroy(goose_ctx* c) {
+    if (!c) return GOOSE_EINVAL;
+    cudaSetDevice(c->device);
+    cudaFree(c->partials); cudaFree(c->head_counters); cudaFree(c->topk_cand);
+    cudaFree(c->row_counters); cudaFree(c->status); cudaFree(c->stage);
+    delete c;
+    return GOOSE_OK;
+}
+
+int goose_set_attn_impl(goose_ctx* c, int impl) {
+    if (!c || impl < GOOSE_ATTN_AUTO || impl > GOOSE_ATTN_UMMA) return GOOSE_EINVAL;
+    c->attn_impl = impl;
+    return GOOSE_OK;
+}
+
+int64_t goose_launch_count(goose_ctx* c) { return c ? c->launches : -1; }
+
+int goose_tree_attn(goose_ctx* c, const void* q, const void* k_cache, const void* v_cache, int64_t kv_rows,
+                    const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
+                    int S, int B, int H, int D, float scale, void* out, float* lse, void* stream) {
+    int rc = check_shape(c, S, B, H, D);
+    if (rc) return rc;
+    if (!q || !k_cache || !v_cache || !row_off || !ctx_len || !parent || !out) return GOOSE_EINVAL;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out)) return GOOSE_EINVAL;
+    if (kv_rows < 1 || kv_rows > 0x7FFFFFFFLL) return GOOSE_EINVAL;
+    if (S == 0) return GOOSE_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int impl = c->attn_impl;
+    if (impl == GOOSE_ATTN_AUTO) impl = goose::auto_attn_impl(c, S, B, H);
+    cudaError_t e;
+    if (impl == GOOSE_ATTN_UMMA)
+        e = goose::launch_tree_attn_umma(c, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_cache,
+                                         (const __nv_bfloat16*)v_cache, kv_rows, row_off, ctx_len, parent, S, B, H,
+                                         scale, (__nv_bfloat16*)out, lse, st);
+    else
+        e = goose::launch_tree_attn_mma(c, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_cache,
+                                        (const __nv_bfloat16*)v_cache, row_off, ctx_len, parent, S, B, H, scale,
+                                        (__nv_bfloat16*)out, lse, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return GOOSE_OK;
+}
+
+int goose_node_topk(goose_ctx* c, const void* logits, int rows, int V, int64_t ldl, int k,
+                    int32_t* argmax, int32_t* topk_ids, float* topk_vals, void* stream) {
+    if (!c || !logits || !argmax || !topk_ids) return GOOSE_EINVAL;
+    if (rows < 0 || rows > c->topk_rows_cap) return GOOSE_EINVAL;
+    if (V < 1 || V > GOOSE_MAX_V || ldl < V || (ldl & 7) != 0 || !aligned16(logits)) return GOOSE_EINVAL;
+    if (k < 1 || k > GOOSE_MAX_K || k > V) return GOOSE_EINVAL;
+    cudaError_t e = goose::launch_node_topk(c, (const __nv_bfloat16*)logits, rows, V, ldl, k, argmax, topk_ids,
+                                            topk_vals, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e);
+    return GOOSE_OK;
+}
+
+int goose_accept(goose_ctx* c, const int32_t* draft_tok, const int32_t* parent, const int32_t* argmax,
+                 int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus, void* stream) {
+    if (!c || !draft_tok || !parent || !argmax || !path || !accept_len || !bonus) return GOOSE_EINVAL;
+    if (S < 0 || S > c->max_S || B < 1 || B > c->max_B) return GOOSE_EINVAL;
+    cudaError_t e = goose::launch_accept(c, draft_tok, parent, argmax, S, B, path, accept_len, bonus,
+                                         static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e);
+    return GOOSE_OK;
+}
+
+int goose_kv_compact(goose_ctx* c, void* k_cache, void* v_cache, int64_t kv_rows,
+                     const int64_t* row_off, const int32_t* ctx_len, const int32_t* path,
+                     const int32_t* accept_len, int S, int B, int H, int D,
+                     int32_t* new_ctx_len, void* stream) {
+    int rc = check_shape(c, S, B, H, D);
+    if (rc) return rc;
+    if (!k_cache || !v_cache || !row_off || !ctx_len || !path || !accept_len || !new_ctx_len) return GOOSE_EINVAL;
+    if (!aligned16(k_cache) || !aligned16(v_cache) || kv_rows < 1) return GOOSE_EINVAL;
+    cudaError_t e = goose::launch_kv_compact(c, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, row_off, ctx_len,
+                                             path, accept_len, S, B, H, new_ctx_len,
+                                             static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e);
+    return GOOSE_OK;
+}
+
+int goose_verify_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
+                      const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
+                      const int32_t* draft_tok, const void* logits, int64_t ldl,
+                      int S, int B, int H, int D, int V, int k, float scale,
+                      void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
+                      int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
+                      void* stream) {
+    // validate everything before enqueueing anything
+    int rc = check_shape(c, S, B, H, D);
+    if (rc) return rc;
+    if (!q || !k_cache || !v_cache || !row_off || !ctx_len || !parent || !draft_tok || !logits || !out ||
+        !argmax || !topk_ids || !path || !accept_len || !bonus || !new_ctx_len)
+        return GOOSE_EINVAL;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out) || !aligned16(logits))
+        return GOOSE_EINVAL;
+    if (V < 1 || V > GOOSE_MAX_V || ldl < V || (ldl & 7) != 0 || k < 1 || k > GOOSE_MAX_K || k > V) return GOOSE_EINVAL;
+    if ((long long)S * B > c->topk_rows_cap || kv_rows < 1 || kv_rows > 0x7FFFFFFFLL) return GOOSE_EINVAL;
+    rc = goose_tree_attn(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, S, B, H, D, scale, out, lse, stream);
+    if (rc) return rc;
+    rc = goose_node_topk(c, logits, S * B, V, ldl, k, argmax, topk_ids, topk_vals, stream);
+    if (rc) return rc;
+    rc = goose_accept(c, draft_tok, parent, argmax, S, B, path, accept_len, bonus, stream);
+    if (rc) return rc;
+    return goose_kv_compact(c, k_cache, v_cache, kv_rows, row_off, ctx_len, path, accept_len, S, B, H, D,
+                            new_ctx_len, stream);
+}
+
+int goose_verify_step_host(goose_ctx* c, void* k_cache, void* v_cache, int64_t kv_rows,
+                           const void* h_q, const void* h_k_new, const void* h_v_new,
+                           const int64_t* h_row_off, const int32_t* h_ctx_len,
+                           const int32_t* h_parent, const int32_t* h_draft_tok, const void* h_logits,
+                           int S, int B, int H, int D, int V, int k, float scale,
+                           void* h_out, int32_t* h_argmax, int32_t* h_topk_ids, float* h_topk_vals,
+                           int32_t* h_path, int32_t* h_accept_len, int32_t* h_bonus,
+                           int32_t* h_new_ctx_len, void* stream) {
+    int rc = check_shape(c, S, B, H, D);
+    if (rc) return rc;
+    if (!k_cache || !v_cache || !h_q || !h_k_new || !h_v_new || !h_row_off || !h_ctx_len || !h_parent ||
+        !h_draft_tok || !h_logits || !h_out || !h_argmax || !h_topk_ids || !h_path || !h_accept_len || !h_bonus ||
+        !h_new_ctx_len)
+        return GOOSE_EINVAL;
+    if (V < 1 || V > GOOSE_MAX_V || (V & 7) != 0 || k < 1 || k > GOOSE_MAX_K || k > V) return GOOSE_EINVAL;
+    if (S == 0) return GOOSE_OK;
+    for (int s = 0; s < S; ++s)
+        if (h_row_off[s] < 0 || h_ctx_len[s] < 0 || h_row_off[s] + h_ctx_len[s] + B > kv_rows) return GOOSE_EINVAL;
+    GOOSE_CUDA(cudaSetDevice(c->device));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    // staging layout (256-byte aligned pieces)
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    const size_t n_q = (size_t)S * B * H * D * 2, rows = (size_t)S * B;
+    size_t off = 0;
+    const size_t o_q = off; off = up(off + n_q);
+    const size_t o_out = off; off = up(off + n_q);
+    const size_t o_logits = off; off = up(off + rows * V * 2);
+    const size_t o_rowoff = off; off = up(off + S * 8);
+    const size_t o_ctx = off; off = up(off + S * 4);
+    const size_t o_parent = off; off = up(off + rows * 4);
+    const size_t o_tok = off; off = up(off + rows * 4);
+    const size_t o_argmax = off; off = up(off + rows * 4);
+    const size_t o_ids = off; off = up(off + rows * k * 4);
+    const size_t o_vals = off; off = up(off + rows * k * 4);
+    const size_t o_path = off; off = up(off + rows * 4);
+    const size_t o_alen = off; off = up(off + S * 4);
+    const size_t o_bonus = off; off = up(off + S * 4);
+    const size_t o_newctx = off; off = up(off + S * 4);
+    if (off > c->stage_bytes) {
+        GOOSE_CUDA(cudaStreamSynchronize(st));
+        if (c->stage) cudaFree(c->stage);
+        c->stage = nullptr; c->stage_bytes = 0;
+        if (cudaMalloc(&c->stage, off) != cudaSuccess) { cudaGetLastError(); return GOOSE_ENOMEM; }
+        c->stage_bytes = off;
+    }
+    char* d = static_cast<char*>(c->stage);
+    const size_t row_bytes = (size_t)H * D * 2;
+    GOOSE_CUDA(cudaMemcpyAsync(d + o_q, h_q, n_q, cudaMemcpyHostToDevice, st));
+    for (int s = 0; s < S; ++s) {
+        size_t dst = (size_t)(h_row_off[s] + h_ctx_len[s]) * row_bytes;
+        GOOSE_CUDA(cudaMemcpyAsync((char*)k_cache + dst, (const char*)h_k_new + (size_t)s * B * row_bytes,
+                                   (size_t)B * row_bytes, cudaMemcpyHostToDevice, st));
+        GOOSE_CUDA(cudaMemcpyAsync((char*)v_cache + dst, (const char*)h_v_new + (size_t)s * B * row_bytes,
+                                   (size_t)B * row_bytes, cudaMemcpyHostToDevice, st));
+    }
+    GOOSE_CUDA(cudaMemcpyAsync(d + o_logits, h_logits, rows * V * 2, cudaMemcpyHostToDevice, st));
+    GOOSE_CUDA(cudaMemcpyAsync(d + o_rowoff, h_row_off, S * 8, cudaMemcpyHostToDevice, st));
+    GOOSE_CUDA(cudaMemcpyAsync(d + o_ctx, h_ctx_len, S * 4, cudaMemcpyHostToDevice, st));
+    GOOSE_CUDA(cudaMemcpyAsync(d + o_parent, h_parent, rows * 4, cudaMemcpyHostToDevice, st));
+    GOOSE_CUDA(cudaMemcpyAsync(d + o_tok, h_draft_tok, rows * 4, cudaMemcpyHostToDevice, st));
+    rc = goose_verify_step(c, d + o_q, k_cache, v_cache, kv_rows, (const int64_t*)(d + o_rowoff),
+                           (const int32_t*)(d + o_ctx), (const int32_t*)(d + o_parent), (const int32_t*)(d + o_tok),
+                           d + o_logits, V, S, B, H, D, V, k, scale, d + o_out, nullptr, (int32_t*)(d + o_argmax),
+                           (int32_t*)(d + o_ids), (float*)(d + o_vals), (int32_t*)(d + o_path),
+                           (int32_t*)(d + o_alen), (int32_t*)(d + o_bonus), (int32_t*)(d + o_newctx), stream);
+    if (rc) return rc;
+    GOOSE_CUDA(cudaMemcpyAsync(h_out, d + o_out, n_q, cudaMemcpyDeviceToHost, st));
+    GOOSE_CUDA(cudaMemcpyAsync(h_argmax, d + o_argmax, rows * 4, cudaMemcpyDeviceToHost, st));
+    GOOSE_CUDA(cudaMemcpyAsync(h_topk_ids, d + o_ids, rows * k * 4, cudaMemcpyDeviceToHost, st));
+    if (h_topk_vals) GOOSE_CUDA(cudaMemcpyAsync(h_topk_vals, d + o_vals, rows * k * 4, cudaMemcpyDeviceToHost, st));
+    GOOSE_CUDA(cudaMemcpyAsync(h_path, d + o_path, rows * 4, cudaMemcpyDeviceToHost, st));
+    GOOSE_CUDA(cudaMemcpyAsync(h_accept_len, d + o_alen, S * 4, cudaMemcpyDeviceToHost, st));
+    GOOSE_CUDA(cudaMemcpyAsync(h_bonus, d + o_bonus, S * 4, cudaMemcpyDeviceToHost, st));
+    GOOSE_CUDA(cudaMemcpyAsync(h_new_ctx_len, d + o_newctx, S * 4, cudaMemcpyDeviceToHost, st));
+    GOOSE_CUDA(cudaStreamSynchronize(st));
+    return GOOSE_OK;
+}
+
+int goose_last_status(goose_ctx* c, int32_t* host_status, int S) {
+    if (!c || !host_status || S < 0 || S > c->max_S) return GOOSE_EINVAL;
+    GOOSE_CUDA(cudaSetDevice(c->device));
+    GOOSE_CUDA(cudaDeviceSynchronize());
+    GOOSE_CUDA(cudaMemcpy(host_status, c->status, sizeof(int32_t) * (size_t)S, cudaMemcpyDeviceToHost));
+    GOOSE_CUDA(cudaMemset(c->status, 0, sizeof(int32_t) * (size_t)c->max_S));
+    int rc = GOOSE_OK;
+    for (int s = 0; s < S; ++s)
+        if (host_status[s] & GOOSE_ST_TIMEOUT) rc = GOOSE_ETIMEOUT;
+    return rc;
+}
+
+}  // extern "C"

@@ -1,0 +1,78 @@
+// Internal declarations shared by the CUDA translation units of libgoose.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "goose.h"
+
+namespace goose {
+
+constexpr int kHeadDim = GOOSE_HEAD_DIM;
+constexpr int kMaxB = GOOSE_MAX_B;
+constexpr int kMaxK = GOOSE_MAX_K;
+
+// Workspace layout of one split-KV partial: O fp32 [kMaxB][128] (unnormalised), then m[kMaxB], l[kMaxB].
+constexpr int kPartialFloats = kMaxB * kHeadDim + 2 * kMaxB;
+
+}  // namespace goose
+
+struct goose_ctx {
+    int device;
+    int num_sms;
+    int max_S, max_B, max_H;
+    int attn_impl;            // GOOSE_ATTN_*
+    // attention workspace
+    float* partials;          // [n_slots][kPartialFloats]
+    int n_slots;
+    int32_t* head_counters;   // [max_S * max_H], zero between launches
+    // top-k workspace
+    unsigned long long* topk_cand;   // [topk_rows_cap][topk_chunks_cap][kMaxK]
+    int32_t* row_counters;    // [topk_rows_cap]
+    int64_t topk_cand_cap;    // elements
+    int topk_rows_cap;
+    // per-sequence status words
+    int32_t* status;          // [max_S]
+    // host staging for goose_verify_step_host
+    void* stage;              // device buffer
+    size_t stage_bytes;
+    long long launches;
+    void* encode_tiled;       // cuTensorMapEncodeTiled entry point (driver), resolved at create
+};
+
+namespace goose {
+
+// launchers (each returns a cudaError_t from the launch)
+cudaError_t launch_node_topk(goose_ctx* c, const __nv_bfloat16* logits, int rows, int V, int64_t ldl, int k,
+                             int32_t* argmax, int32_t* ids, float* vals, cudaStream_t st);
+cudaError_t launch_accept(goose_ctx* c, const int32_t* draft_tok, const int32_t* parent, const int32_t* argmax,
+                          int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus, cudaStream_t st);
+cudaError_t launch_kv_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* row_off,
+                              const int32_t* ctx_len, const int32_t* path, const int32_t* accept_len,
+                              int S, int B, int H, int32_t* new_ctx, cudaStream_t st);
+cudaError_t launch_tree_attn_mma(goose_ctx* c, const __nv_bfloat16* q, const __nv_bfloat16* kc,
+                                 const __nv_bfloat16* vc, const int64_t* row_off, const int32_t* ctx_len,
+                                 const int32_t* parent, int S, int B, int H, float scale,
+                                 __nv_bfloat16* out, float* lse, cudaStream_t st);
+cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __nv_bfloat16* kc,
+                                  const __nv_bfloat16* vc, int64_t kv_rows, const int64_t* row_off,
+                                  const int32_t* ctx_len, const int32_t* parent, int S, int B, int H,
+                                  float scale, __nv_bfloat16* out, float* lse, cudaStream_t st);
+
+// Max context rows assumed when sizing the fixed-split grid of the mma kernel is not needed:
+// ctx_len lives on the device, so the split count depends only on S, H and the SM count.
+int mma_splits(const goose_ctx* c, int S, int H);
+
+// per-device kernel attributes (dynamic shared memory limits); called once from goose_create
+cudaError_t init_mma_kernel();
+cudaError_t init_umma_kernel();
+inline cudaError_t init_kernels(goose_ctx*) {
+    cudaError_t e = init_mma_kernel();
+    return e != cudaSuccess ? e : init_umma_kernel();
+}
+
+// kernel choice of GOOSE_ATTN_AUTO
+int auto_attn_impl(const goose_ctx* c, int S, int B, int H);
+
+}  // namespace goose

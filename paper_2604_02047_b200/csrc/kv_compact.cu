@@ -1,0 +1,77 @@
+// In-place KV compaction of the accepted path (the paper leaves cache handling after acceptance
+// implicit; the accepted nodes' rows are kept, in path order, directly after the prefix).
+//
+// Row ctx+j <- row ctx+path[j].  path is increasing with path[j] >= j, so a thread that owns one
+// 16-byte column of the row and walks j upwards never overwrites a row it still has to read:
+// sources of later moves are > j.  Moves are issued in batches of 8 (all loads of a batch before its
+// stores; a batch's destinations are below every later source), which keeps 8 loads in flight per
+// thread without any barrier.
+#include "goose_internal.cuh"
+
+namespace goose {
+
+constexpr int kCompactThreads = 128;
+constexpr int kCompactBatch = 8;
+
+__global__ void __launch_bounds__(kCompactThreads)
+kv_compact_kernel(__nv_bfloat16* __restrict__ kc, __nv_bfloat16* __restrict__ vc,
+                  const int64_t* __restrict__ row_off, const int32_t* __restrict__ ctx_len,
+                  const int32_t* __restrict__ path, const int32_t* __restrict__ accept_len,
+                  int B, int row_vec /* 16-byte vectors per row = H*128*2/16 */,
+                  int32_t* __restrict__ new_ctx, int32_t* __restrict__ status) {
+    __shared__ int s_path[kMaxB];
+    __shared__ int s_bad;
+    const int s = blockIdx.z;
+    const int which = blockIdx.y;                        // 0 = K, 1 = V
+    const int col = blockIdx.x * kCompactThreads + threadIdx.x;
+    const int ctx = ctx_len[s];
+    int L = accept_len[s];
+    if (threadIdx.x == 0) s_bad = 0;
+    __syncthreads();
+    bool bad = (L < 0 || L >= B);
+    if (!bad) {
+        for (int j = threadIdx.x; j <= L; j += kCompactThreads) {
+            int pj = path[(size_t)s * B + j];
+            s_path[j] = pj;
+            int prev = (j == 0) ? -1 : path[(size_t)s * B + j - 1];
+            if (pj < j || pj >= B || pj <= prev || (j == 0 && pj != 0)) s_bad = 1;
+        }
+    }
+    __syncthreads();
+    bad = bad || s_bad;
+    if (bad) L = 0;
+    if (blockIdx.x == 0 && which == 0 && threadIdx.x == 0) {
+        new_ctx[s] = ctx + 1 + L;
+        if (bad) atomicOr(&status[s], GOOSE_ST_BAD_PATH);
+    }
+    if (bad || col >= row_vec) return;
+
+    uint4* base = reinterpret_cast<uint4*>(which ? vc : kc) + ((size_t)(row_off[s] + ctx)) * row_vec + col;
+    for (int j0 = 1; j0 <= L; j0 += kCompactBatch) {
+        uint4 r[kCompactBatch];
+#pragma unroll
+        for (int t = 0; t < kCompactBatch; ++t) {
+            int j = j0 + t;
+            if (j <= L && s_path[j] != j) r[t] = base[(size_t)s_path[j] * row_vec];
+        }
+#pragma unroll
+        for (int t = 0; t < kCompactBatch; ++t) {
+            int j = j0 + t;
+            if (j <= L && s_path[j] != j) base[(size_t)j * row_vec] = r[t];
+        }
+    }
+}
+
+cudaError_t launch_kv_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* row_off,
+                              const int32_t* ctx_len, const int32_t* path, const int32_t* accept_len,
+                              int S, int B, int H, int32_t* new_ctx, cudaStream_t st) {
+    if (S == 0) return cudaSuccess;
+    int row_vec = H * kHeadDim * 2 / 16;
+    dim3 grid((row_vec + kCompactThreads - 1) / kCompactThreads, 2, S);
+    kv_compact_kernel<<<grid, kCompactThreads, 0, st>>>(kc, vc, row_off, ctx_len, path, accept_len, B, row_vec,
+                                                        new_ctx, c->status);
+    c->launches++;
+    return cudaGetLastError();
+}
+
+}  // namespace goose

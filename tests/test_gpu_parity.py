@@ -1,0 +1,324 @@
+"""GPU parity: every call goes through the C ABI and is compared with the fp64 oracle on the same
+seeded inputs.  Integer results (argmax, top-k ids, path, lengths, cache rows) must be bit-exact;
+attention must satisfy, per (sequence, node, head) row, max_d |gpu - ref| <= 1e-2 * max_d |ref|
+(bf16 inputs, fp32 accumulation, bf16 output)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2604_02047_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+ATTN_TOL = 1e-2
+
+
+@pytest.fixture(scope="module")
+def goose():
+    from paper_2604_02047_b200 import binding, build
+    build.build()
+    g = binding.Goose(max_S=16, max_B=128, max_H=64)
+    yield g
+    g.close()
+
+
+def _impls():
+    from paper_2604_02047_b200 import binding
+    return [binding.ATTN_MMA, binding.ATTN_UMMA]
+
+
+def _impl_ids():
+    return ["mma", "umma"]
+
+
+def attn_row_err(gpu_out, ref_out):
+    """gpu_out, ref_out: [..., D] float64.  Returns the per-row normalised max error."""
+    num = np.abs(gpu_out - ref_out).max(axis=-1)
+    den = np.abs(ref_out).max(axis=-1)
+    return num / den
+
+
+def _run_attn(goose, x, impl, want_lse=True):
+    from paper_2604_02047_b200 import binding
+    goose.set_attn_impl(impl)
+    d = binding.to_device(x)
+    out, lse = goose.tree_attn(d["q"], d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], d["parent"],
+                               x.scale, want_lse=want_lse)
+    torch.cuda.synchronize()
+    st = goose.last_status(x.S)
+    goose.set_attn_impl(binding.ATTN_AUTO)
+    return out.float().cpu().numpy().astype(np.float64), (lse.cpu().numpy().astype(np.float64) if want_lse else None), st
+
+
+def _check_attn_full(goose, oracle, x, impl):
+    out, lse, st = _run_attn(goose, x, impl)
+    assert not st.any()
+    ref, ref_lse = oracle.tree_attn(x.q, x.k_cache, x.v_cache, x.row_off, x.ctx_len, x.parent, x.scale)
+    err = attn_row_err(out, ref)
+    assert err.max() <= ATTN_TOL, (err.max(), np.unravel_index(err.argmax(), err.shape))
+    assert np.abs(lse - ref_lse).max() <= 2e-3
+
+
+# ------------------------------------------------------------------ attention
+@pytest.mark.parametrize("impl", _impls(), ids=_impl_ids())
+@pytest.mark.parametrize("ctx", [0, 1, 127, 128, 129, 300])
+@pytest.mark.parametrize("B,tree", [(1, "chain"), (2, "chain"), (16, "spine"), (17, "random"), (64, "kary3"),
+                                     (80, "spine"), (128, "kary5"), (128, "chain"), (33, "star")])
+def test_attention_fixture_shapes(goose, oracle, impl, ctx, B, tree):
+    rng = np.random.default_rng([ctx, B, 5])
+    par = {"chain": lambda: synth.chain_tree(B), "star": lambda: synth.star_tree(B),
+           "kary3": lambda: synth.kary_tree(B, 3), "kary5": lambda: synth.kary_tree(B, 5),
+           "random": lambda: synth.random_tree(rng, B),
+           "spine": lambda: synth.spine_tree(rng, B, max(1, B // 4), 3)[0]}[tree]()
+    x = synth.make_inputs(1, 3, B, [ctx], [par], V=8, with_logits=False, seed=ctx * 131 + B)
+    _check_attn_full(goose, oracle, x, impl)
+
+
+@pytest.mark.parametrize("impl", _impls(), ids=_impl_ids())
+def test_attention_ragged_batch_and_peaked_scores(goose, oracle, impl):
+    rng = np.random.default_rng(17)
+    S, B, H = 5, 24, 4
+    ctxs = [700, 0, 129, 1023, 64]
+    parents = [synth.spine_tree(rng, B, 6, 3)[0] for _ in range(S)]
+    x = synth.make_inputs(S, H, B, ctxs, parents, V=8, with_logits=False, seed=23)
+    _check_attn_full(goose, oracle, x, impl)
+    # peaked scores (queries x8): the running max moves a lot, exercising the rescaling path
+    y = synth.make_inputs(2, 2, 40, [900, 257], [synth.random_tree(rng, 40), synth.chain_tree(40)], V=8,
+                          with_logits=False, seed=29, q_gain=8.0)
+    _check_attn_full(goose, oracle, y, impl)
+
+
+@pytest.mark.parametrize("impl", _impls(), ids=_impl_ids())
+def test_attention_never_reads_rows_past_the_tree(goose, oracle, impl):
+    """Rows behind ctx+B (slack, or another sequence's rows) may hold anything, NaN included."""
+    from paper_2604_02047_b200 import binding
+    B, H, ctx = 20, 2, 150
+    x = synth.make_inputs(1, H, B, [ctx], [synth.kary_tree(B, 3)], V=8, with_logits=False, seed=31)
+    pad = np.full((300, H, 128), 0x7FC0, np.uint16)            # bf16 NaN
+    kc = np.concatenate([x.k_cache, pad]); vc = np.concatenate([x.v_cache, pad])
+    goose.set_attn_impl(impl)
+    bf = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).cuda()
+    d = binding.to_device(x)
+    out, _ = goose.tree_attn(d["q"], bf(kc), bf(vc), d["row_off"], d["ctx_len"], d["parent"], x.scale)
+    goose.set_attn_impl(binding.ATTN_AUTO)
+    ref, _ = oracle.tree_attn(x.q, x.k_cache, x.v_cache, x.row_off, x.ctx_len, x.parent, x.scale)
+    got = out.float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert attn_row_err(got, ref).max() <= ATTN_TOL
+
+
+@pytest.mark.parametrize("impl", _impls(), ids=_impl_ids())
+def test_attention_invalid_parent_sets_status_and_zero_fills(goose, impl):
+    B = 12
+    x = synth.make_inputs(2, 2, B, [70, 40], [synth.chain_tree(B), synth.chain_tree(B)], V=8, with_logits=False)
+    x.parent[1, 5] = 7                                         # parent[i] >= i
+    out, lse, st = _run_attn(goose, x, impl)
+    assert st.tolist() == [0, 1]
+    assert np.all(out[1] == 0) and np.abs(out[0]).max() > 0
+
+
+@pytest.mark.parametrize("impl", _impls(), ids=_impl_ids())
+def test_attention_is_deterministic(goose, impl):
+    x = synth.make_config(0, with_logits=False)
+    a, _, _ = _run_attn(goose, x, impl)
+    b, _, _ = _run_attn(goose, x, impl)
+    assert np.array_equal(a, b)
+
+
+# ------------------------------------------------------------------ top-k
+def _check_topk(goose, oracle, bits, k, V=None):
+    lg = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).cuda()
+    am, ids, vals = goose.node_topk(lg, k, V=V)
+    ram, rids, rvals = oracle.node_topk(bits, k, V=V)
+    assert np.array_equal(am.cpu().numpy(), ram)
+    assert np.array_equal(ids.cpu().numpy(), rids)
+    assert np.array_equal(vals.cpu().numpy().astype(np.float64), rvals)
+
+
+def test_topk_generator_logits_and_ties(goose, oracle):
+    x = synth.make_config(0)
+    _check_topk(goose, oracle, x.logits, 8)
+    rng = np.random.default_rng(0)
+    coarse = synth.f32_to_bf16_bits((np.round(rng.standard_normal((64, 32000)) * 2) / 2).astype(np.float32))
+    _check_topk(goose, oracle, coarse, 8)
+    _check_topk(goose, oracle, coarse, 16)
+    _check_topk(goose, oracle, coarse, 1)
+
+
+@pytest.mark.parametrize("V,ldl,k", [(1, 8, 1), (5, 8, 5), (100, 104, 8), (8191, 8192, 8), (8192, 8192, 16),
+                                      (8193, 8200, 8), (32001, 32008, 10), (151936, 151936, 16)])
+def test_topk_sizes(goose, oracle, V, ldl, k):
+    rng = np.random.default_rng(V)
+    bits = synth.f32_to_bf16_bits(rng.standard_normal((7, ldl), dtype=np.float32))
+    bits[:, V:] = 0x7F00                                       # huge values in the padding must be ignored
+    _check_topk(goose, oracle, bits, k, V=V)
+
+
+def test_topk_special_rows(goose, oracle):
+    V = 32000
+    rows = np.zeros((6, V), np.uint16)
+    rows[0, :] = 0x4000                                        # constant row -> ids 0..k-1
+    rows[1, ::2] = 0x8000                                      # -0.0 / +0.0 mix: all equal
+    rows[2] = synth.f32_to_bf16_bits(np.linspace(-3, 3, V, dtype=np.float32)); rows[2, 0] = rows[2, V - 1]
+    rows[3] = synth.f32_to_bf16_bits(-np.arange(1, V + 1, dtype=np.float32))
+    rows[4, :] = 0xC000; rows[4, V - 1] = 0x0000               # all -2 except the last
+    rows[5, :] = 0xFF7F                                        # most negative finite bf16 everywhere
+    _check_topk(goose, oracle, rows, 8)
+
+
+# ------------------------------------------------------------------ accept
+def test_accept_random_trees(goose, oracle):
+    rng = np.random.default_rng(3)
+    for B in (1, 2, 7, 32, 33, 64, 100, 128):
+        S = 16
+        parent = np.stack([synth.random_tree(rng, B) if s % 2 else synth.spine_tree(rng, B, max(1, B // 3), 3)[0]
+                           for s in range(S)])
+        tok = np.stack([synth.distinct_sibling_tokens(rng, parent[s], 6) for s in range(S)])
+        am = rng.integers(0, 6, size=(S, B)).astype(np.int32)
+        if B > 2:
+            am[0, :-1] = tok[0, 1:] if np.all(parent[0][1:] == np.arange(B - 1)) else am[0, :-1]
+        p, l, b = goose.accept(torch.from_numpy(tok).cuda(), torch.from_numpy(parent).cuda(), torch.from_numpy(am).cuda())
+        rp, rl, rb = oracle.accept(tok, parent, am)
+        assert np.array_equal(p.cpu().numpy(), rp) and np.array_equal(l.cpu().numpy(), rl)
+        assert np.array_equal(b.cpu().numpy(), rb)
+
+
+def test_accept_full_chain_duplicates_and_invalid(goose, oracle):
+    B = 128
+    parent = synth.chain_tree(B)[None]
+    tok = np.arange(100, 100 + B, dtype=np.int32)[None]
+    am = np.concatenate([tok[0, 1:], [42]]).astype(np.int32)[None]
+    p, l, b = goose.accept(torch.from_numpy(tok).cuda(), torch.from_numpy(parent).cuda(), torch.from_numpy(am).cuda())
+    assert l.item() == B - 1 and b.item() == 42 and p.cpu().numpy()[0].tolist() == list(range(B))
+    parent = np.array([[-1, 0, 0, 0]], np.int32); tok = np.array([[1, 5, 5, 5]], np.int32)
+    am = np.array([[5, 9, 8, 7]], np.int32)
+    p, l, b = goose.accept(torch.from_numpy(tok).cuda(), torch.from_numpy(parent).cuda(), torch.from_numpy(am).cuda())
+    rp, rl, rb = oracle.accept(tok, parent, am)
+    assert np.array_equal(p.cpu().numpy(), rp) and l.item() == rl[0] and b.item() == rb[0]
+    bad = np.array([[-1, 0, 3, 1], [-1, 0, 1, 2]], np.int32)
+    z = torch.zeros((2, 4), dtype=torch.int32).cuda()
+    p, l, b = goose.accept(z, torch.from_numpy(bad).cuda(), z)
+    st = goose.last_status(2)
+    assert st.tolist() == [1, 0] and l.cpu().tolist()[0] == 0 and b.cpu().tolist()[0] == -1
+    assert p.cpu().numpy()[0].tolist() == [0, -1, -1, -1]
+
+
+# ------------------------------------------------------------------ compaction
+def test_kv_compact_random_paths(goose, oracle):
+    from paper_2604_02047_b200 import binding
+    rng = np.random.default_rng(9)
+    S, B, H = 6, 40, 5
+    parents = [synth.random_tree(rng, B) if s % 2 else synth.chain_tree(B) for s in range(S)]
+    x = synth.make_inputs(S, H, B, [33, 0, 200, 1, 64, 17], parents, V=8, with_logits=False, seed=6)
+    path = np.full((S, B), -1, np.int32); alen = np.zeros(S, np.int32)
+    for s in range(S):
+        v, L = 0, 0
+        path[s, 0] = 0
+        while True:
+            kids = [c for c in range(B) if parents[s][c] == v]
+            if not kids or (s != 2 and rng.random() < 0.1):
+                break
+            v = int(rng.choice(kids)); L += 1; path[s, L] = v
+        alen[s] = L
+    assert alen[2] == B - 1                                    # a fully accepted chain
+    d = binding.to_device(x)
+    new_ctx = goose.kv_compact(d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"],
+                               torch.from_numpy(path).cuda(), torch.from_numpy(alen).cuda())
+    rk, rv, rn = oracle.kv_compact(x.k_cache, x.v_cache, x.row_off, x.ctx_len, path, alen)
+    assert np.array_equal(new_ctx.cpu().numpy(), rn)
+    gk, gv = binding.bf16_to_bits(d["k_cache"]), binding.bf16_to_bits(d["v_cache"])
+    for s in range(S):
+        r0, n = int(x.row_off[s]), int(rn[s])
+        assert np.array_equal(gk[r0:r0 + n], rk[r0:r0 + n]) and np.array_equal(gv[r0:r0 + n], rv[r0:r0 + n])
+    assert not goose.last_status(S).any()
+
+
+def test_kv_compact_invalid_path_is_flagged(goose):
+    from paper_2604_02047_b200 import binding
+    x = synth.make_inputs(2, 2, 8, [10, 10], [synth.chain_tree(8)] * 2, V=8, with_logits=False)
+    d = binding.to_device(x)
+    before = binding.bf16_to_bits(d["k_cache"]).copy()
+    path = torch.tensor([[0, 3, 2, -1, -1, -1, -1, -1], [0, 1, 2, -1, -1, -1, -1, -1]], dtype=torch.int32).cuda()
+    alen = torch.tensor([2, 2], dtype=torch.int32).cuda()
+    new_ctx = goose.kv_compact(d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], path, alen)
+    assert goose.last_status(2).tolist() == [2, 0]
+    assert new_ctx.cpu().tolist() == [11, 13]
+    assert np.array_equal(binding.bf16_to_bits(d["k_cache"])[:18], before[:18])   # sequence 0 untouched
+
+
+# ------------------------------------------------------------------ whole step on the benchmark configs
+def _check_step(goose, oracle, x, n_rows=192, host=False):
+    from paper_2604_02047_b200 import binding
+    d = binding.to_device(x)
+    if host:
+        houts = goose.alloc_step_outputs(x.S, x.B, x.H, x.D, x.k, device="cpu")
+        houts = {k_: v.pin_memory() for k_, v in houts.items()}
+        hin = {k_: v.cpu().pin_memory() for k_, v in d.items()}
+        rows = np.concatenate([np.arange(x.row_off[s] + x.ctx_len[s], x.row_off[s] + x.ctx_len[s] + x.B) for s in range(x.S)])
+        rows_t = torch.from_numpy(rows).cuda()
+        k_new = d["k_cache"][rows_t].reshape(x.S, x.B, x.H, x.D).cpu().pin_memory()
+        v_new = d["v_cache"][rows_t].reshape(x.S, x.B, x.H, x.D).cpu().pin_memory()
+        d["k_cache"][rows_t] = 0; d["v_cache"][rows_t] = 0     # the call must put the tree rows in place itself
+        o = goose.verify_step_host(d["k_cache"], d["v_cache"], hin["q"], k_new, v_new, hin["row_off"], hin["ctx_len"],
+                                   hin["parent"], hin["draft_tok"], hin["logits"], x.k, x.scale, houts)
+    else:
+        o = goose.verify_step(d["q"], d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], d["parent"],
+                              d["draft_tok"], d["logits"], x.k, x.scale)
+        torch.cuda.synchronize()
+    assert not goose.last_status(x.S).any()
+    ram, rids, rvals = oracle.node_topk(x.logits, x.k)
+    rp, rl, rb = oracle.accept(x.draft_tok, x.parent, ram.reshape(x.S, x.B))
+    rk, rv, rn = oracle.kv_compact(x.k_cache, x.v_cache, x.row_off, x.ctx_len, rp, rl)
+    assert np.array_equal(o["argmax"].cpu().numpy(), ram) and np.array_equal(o["topk_ids"].cpu().numpy(), rids)
+    assert np.array_equal(o["topk_vals"].cpu().numpy().astype(np.float64), rvals)
+    assert np.array_equal(o["path"].cpu().numpy(), rp) and np.array_equal(o["accept_len"].cpu().numpy(), rl)
+    assert np.array_equal(o["bonus"].cpu().numpy(), rb) and np.array_equal(o["new_ctx_len"].cpu().numpy(), rn)
+    gk, gv = binding.bf16_to_bits(d["k_cache"]), binding.bf16_to_bits(d["v_cache"])
+    for s in range(x.S):
+        r0, n = int(x.row_off[s]), int(rn[s])
+        assert np.array_equal(gk[r0:r0 + n], rk[r0:r0 + n]) and np.array_equal(gv[r0:r0 + n], rv[r0:r0 + n])
+    # attention: sampled (sequence, node, head) rows, always including node 0, the deepest node and the last node
+    rng = np.random.default_rng(1)
+    ss = rng.integers(0, x.S, n_rows); si = rng.integers(0, x.B, n_rows); sh = rng.integers(0, x.H, n_rows)
+    si[:3] = [0, x.B - 1, int(np.argmax(x.is_spine[ss[2]].cumsum() * x.is_spine[ss[2]]))]
+    ref, _ = oracle.tree_attn_rows(x.q, x.k_cache, x.v_cache, x.row_off, x.ctx_len, x.parent, x.scale, ss, si, sh)
+    got = o["out"].float().cpu().numpy().astype(np.float64)[ss, si, sh]
+    err = attn_row_err(got, ref)
+    assert err.max() <= ATTN_TOL, err.max()
+    return float(err.max())
+
+
+@pytest.mark.parametrize("config_id", [0, 1, 2, 3, 4])
+def test_verify_step_on_benchmark_configs(goose, oracle, config_id):
+    x = synth.make_config(config_id, seed=0)
+    _check_step(goose, oracle, x)
+
+
+def test_verify_step_full_attention_check_tiny(goose, oracle):
+    x = synth.make_config(0, seed=1)
+    from paper_2604_02047_b200 import binding
+    for impl in _impls():
+        _check_attn_full(goose, oracle, x, impl)
+
+
+def test_verify_step_host_buffers(goose, oracle):
+    _check_step(goose, oracle, synth.make_config(0, seed=2), host=True)
+    _check_step(goose, oracle, synth.make_inputs(3, 4, 16, [100, 7, 260],
+                                                 [synth.kary_tree(16, 3), synth.chain_tree(16), synth.star_tree(16)],
+                                                 V=1024, seed=3), host=True)
+
+
+def test_host_side_argument_errors(goose):
+    from paper_2604_02047_b200 import binding
+    x = synth.make_config(0)
+    d = binding.to_device(x)
+    with pytest.raises(binding.GooseError):
+        goose.node_topk(d["logits"], 17)                       # k > 16
+    with pytest.raises(binding.GooseError):
+        goose.node_topk(d["logits"][:, :31999].contiguous(), 8)  # ldl % 8 != 0
+    with pytest.raises(binding.GooseError):
+        goose.tree_attn(d["q"][..., :64].contiguous(), d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"],
+                        d["parent"], x.scale)                  # head_dim != 128
+    q_mis = torch.empty(x.q.size + 4, dtype=torch.bfloat16, device="cuda")[4:].view(x.q.shape)
+    with pytest.raises(binding.GooseError):
+        goose.tree_attn(q_mis, d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], d["parent"], x.scale)

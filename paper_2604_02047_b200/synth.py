@@ -136,6 +136,8 @@ def random_tree(rng: np.random.Generator, B: int) -> np.ndarray:
 def distinct_sibling_tokens(rng: np.random.Generator, parent: np.ndarray, V: int) -> np.ndarray:
     """Draft tokens uniform in [0, V), redrawn until distinct among siblings."""
     B = len(parent)
+    if B > 1 and int(np.bincount(np.asarray(parent[1:], dtype=np.int64)).max()) > V:
+        raise ValueError("a node has more children than there are tokens")
     tok = rng.integers(0, V, size=B).astype(np.int32)
     seen: Dict[int, set] = {}
     for i in range(B):
@@ -236,7 +238,7 @@ def make_inputs(S: int, H: int, B: int, ctx_lens, parents, *, V: int = VOCAB, k:
         q[s] = f32_to_bf16_bits(qf)
         kc[r0:r0 + n] = normal_bf16(_rng(seed, config_id, s, _ST_K), (n, H, D))
         vc[r0:r0 + n] = normal_bf16(_rng(seed, config_id, s, _ST_V), (n, H, D))
-        tok[s] = distinct_sibling_tokens(_rng(seed, config_id, s, _ST_TOK), parents[s], V)
+        tok[s] = distinct_sibling_tokens(_rng(seed, config_id, s, _ST_TOK), parents[s], V if with_logits else max(V, 4096))
         if with_logits:
             bits, pl = planted_logits(_rng(seed, config_id, s, _ST_LOGIT), _rng(seed, config_id, s, _ST_PLANT),
                                       parents[s], is_spine[s], tok[s], V, float(p_sp[s]), p_branch)

@@ -1,0 +1,45 @@
+"""The N > 1 plumbing of bench.py (replicas only: barrier + max-over-ranks timing), on CPU with gloo."""
+import os
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, q):
+    sys.path.insert(0, ROOT)
+    import bench
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    local_ms = 10.0 if rank == 0 else 25.0                      # rank 1 is the slow one
+    bench.dist_barrier()
+    value, ms_per_step = bench.aggregate_steps_per_s(50, local_ms, world, torch.device("cpu"))
+    q.put((rank, value, ms_per_step, bench.dist_max(float(rank), torch.device("cpu"))))
+    dist.destroy_process_group()
+
+
+def test_two_rank_aggregate_uses_the_slowest_rank():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 29500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in range(2))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, value, ms_per_step, mx in res:
+        assert abs(value - 2 * 50 / 0.025) < 1e-6 and abs(ms_per_step - 0.5) < 1e-9 and mx == 1.0
+
+
+def test_single_process_is_a_noop():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.dist_max(3.5, torch.device("cpu")) == 3.5
+    v, ms = bench.aggregate_steps_per_s(10, 5.0, 1, torch.device("cpu"))
+    assert abs(v - 2000.0) < 1e-9 and abs(ms - 0.5) < 1e-12

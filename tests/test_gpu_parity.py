@@ -41,12 +41,14 @@ def attn_row_err(gpu_out, ref_out):
 def _run_attn(goose, x, impl, want_lse=True):
     from paper_2604_02047_b200 import binding
     goose.set_attn_impl(impl)
-    d = binding.to_device(x)
-    out, lse = goose.tree_attn(d["q"], d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], d["parent"],
-                               x.scale, want_lse=want_lse)
-    torch.cuda.synchronize()
-    st = goose.last_status(x.S)
-    goose.set_attn_impl(binding.ATTN_AUTO)
+    try:
+        d = binding.to_device(x)
+        out, lse = goose.tree_attn(d["q"], d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], d["parent"],
+                                   x.scale, want_lse=want_lse)
+        torch.cuda.synchronize()
+        st = goose.last_status(x.S)
+    finally:
+        goose.set_attn_impl(binding.ATTN_AUTO)
     return out.float().cpu().numpy().astype(np.float64), (lse.cpu().numpy().astype(np.float64) if want_lse else None), st
 
 
@@ -99,8 +101,11 @@ def test_attention_never_reads_rows_past_the_tree(goose, oracle, impl):
     goose.set_attn_impl(impl)
     bf = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).cuda()
     d = binding.to_device(x)
-    out, _ = goose.tree_attn(d["q"], bf(kc), bf(vc), d["row_off"], d["ctx_len"], d["parent"], x.scale)
-    goose.set_attn_impl(binding.ATTN_AUTO)
+    try:
+        out, _ = goose.tree_attn(d["q"], bf(kc), bf(vc), d["row_off"], d["ctx_len"], d["parent"], x.scale)
+        torch.cuda.synchronize()
+    finally:
+        goose.set_attn_impl(binding.ATTN_AUTO)
     ref, _ = oracle.tree_attn(x.q, x.k_cache, x.v_cache, x.row_off, x.ctx_len, x.parent, x.scale)
     got = out.float().cpu().numpy().astype(np.float64)
     assert np.isfinite(got).all()
@@ -173,12 +178,16 @@ def test_accept_random_trees(goose, oracle):
         S = 16
         parent = np.stack([synth.random_tree(rng, B) if s % 2 else synth.spine_tree(rng, B, max(1, B // 3), 3)[0]
                            for s in range(S)])
-        tok = np.stack([synth.distinct_sibling_tokens(rng, parent[s], 6) for s in range(S)])
-        am = rng.integers(0, 6, size=(S, B)).astype(np.int32)
-        if B > 2:
-            am[0, :-1] = tok[0, 1:] if np.all(parent[0][1:] == np.arange(B - 1)) else am[0, :-1]
+        tok = np.stack([synth.distinct_sibling_tokens(rng, parent[s], 1000) for s in range(S)])
+        am = rng.integers(0, 1000, size=(S, B)).astype(np.int32)
+        for s in range(S):                                     # most nodes predict one of their children
+            for v in range(B):
+                kids = np.nonzero(parent[s] == v)[0]
+                if len(kids) and rng.random() < 0.8:
+                    am[s, v] = tok[s, rng.choice(kids)]
         p, l, b = goose.accept(torch.from_numpy(tok).cuda(), torch.from_numpy(parent).cuda(), torch.from_numpy(am).cuda())
         rp, rl, rb = oracle.accept(tok, parent, am)
+        assert rl.max() >= min(B - 1, 2)
         assert np.array_equal(p.cpu().numpy(), rp) and np.array_equal(l.cpu().numpy(), rl)
         assert np.array_equal(b.cpu().numpy(), rb)
 

@@ -80,8 +80,8 @@ def test_source_priority_never_changes_the_path_with_distinct_siblings(oracle):
     for trial in range(100):
         B = 12
         parent, is_spine = synth.spine_tree(rng, B, 5, 2)
-        tok = synth.distinct_sibling_tokens(rng, parent, 6)
-        am = rng.integers(0, 6, size=B).astype(np.int32)
+        tok = synth.distinct_sibling_tokens(rng, parent, 16)
+        am = rng.integers(0, 16, size=B).astype(np.int32)
         a = oracle.accept(tok, parent, am)
         b = oracle.accept(tok, parent, am, tag=is_spine[None])
         assert all(np.array_equal(u, v) for u, v in zip(a, b))

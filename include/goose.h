@@ -86,7 +86,7 @@ int goose_set_attn_impl(goose_ctx* ctx, int impl);
  *   row_off  int64 [S], ctx_len int32 [S], parent int32 [S][B]   (device arrays)
  *   out      bf16 [S][B][H][D]; lse fp32 [S][B][H] = log-sum-exp of the scaled scores, or NULL
  * Rows row_off[s]+ctx_len[s]+B .. are never read as values (their contents may be anything).
- * ctx_len[s] = 0 is legal.  S <= max_S, B <= max_B, H <= max_H, D == 128.                       */
+ * ctx_len[s] = 0 is legal.  S <= max_S, B <= max_B, H <= max_H, D == 128, 0 < scale < 1e30.       */
 int goose_tree_attn(goose_ctx* ctx, const void* q, const void* k_cache, const void* v_cache, int64_t kv_rows,
                     const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
                     int S, int B, int H, int D, float scale, void* out, float* lse, void* stream);

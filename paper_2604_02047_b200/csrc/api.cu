@@ -31,8 +31,8 @@ int check_shape(const goose_ctx* c, int S, int B, int H, int D) {
     return GOOSE_OK;
 }
 
-constexpr int kTopkChunkElems = 8192;
-constexpr int kTopkMaxChunks = GOOSE_MAX_V / kTopkChunkElems;   // 32
+constexpr int kTopkChunkElems = 32768;
+constexpr int kTopkMaxChunks = GOOSE_MAX_V / kTopkChunkElems;   // 8
 
 }  // namespace
 
@@ -133,6 +133,7 @@ int goose_tree_attn(goose_ctx* c, const void* q, const void* k_cache, const void
     if (!q || !k_cache || !v_cache || !row_off || !ctx_len || !parent || !out) return GOOSE_EINVAL;
     if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out)) return GOOSE_EINVAL;
     if (kv_rows < 1 || kv_rows > 0x7FFFFFFFLL) return GOOSE_EINVAL;
+    if (!(scale > 0.f) || !(scale < 1e30f)) return GOOSE_EINVAL;
     if (S == 0) return GOOSE_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int impl = c->attn_impl;

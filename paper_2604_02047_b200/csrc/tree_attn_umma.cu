@@ -1,9 +1,667 @@
-// placeholder until the tcgen05 kernel lands
+// Tree attention on the 5th-generation tensor cores: persistent, warp-specialised kernel
+// (tcgen05.mma with TMEM accumulators, TMA loads, mbarrier pipeline).
+//
+// Work = all (sequence, head, 128-key tile) items in sequence-major order, dealt to the CTAs
+// (one per SM) in contiguous ranges, so every SM streams the same number of K/V bytes.  A run of
+// items of one head inside a CTA's range is a "segment"; a segment that covers its whole head
+// writes the bf16 output directly, any other segment writes an fp32 partial (unnormalised O, running
+// max m, running sum l) and the last CTA to arrive for the head (arrival counter, no spinning)
+// combines the partials.
+//
+// Roles (192 threads):
+//   warp 0, lane 0   TMA producer: Q of the segment, then K and V tiles into a ring of 32 KB stages
+//   warp 1, lane 0   MMA issuer:   S = Q K^T into TMEM (double buffered), O += P V into TMEM
+//   warps 2..5       softmax:      one query row per thread (TMEM lane = row): S from TMEM, ancestor
+//                                  mask on the tiles that reach the tree rows, exp2, P (bf16) into
+//                                  shared memory in the canonical 128-byte-swizzled K-major layout,
+//                                  lazy rescaling of O in TMEM, epilogue / partial / combine.
+// All B <= 128 query rows ride in one M = 128 MMA; rows >= B compute on don't-care data and are
+// never written out.  The tree part of the mask (Sec. 4 Stage 1: a node attends to the prefix and to
+// its root-to-node ancestors) is a per-row 128-bit ancestor set built from parent[].
+//
+// Every wait in this file is bounded: when a wait runs out of polls the CTA raises an abort flag,
+// sets GOOSE_ST_TIMEOUT, drains its own copies in flight (again bounded), frees its TMEM and returns.
+#include <cuda.h>
+
 #include "goose_internal.cuh"
+
 namespace goose {
-cudaError_t init_umma_kernel() { return cudaSuccess; }
-int auto_attn_impl(const goose_ctx*, int, int, int) { return GOOSE_ATTN_MMA; }
-cudaError_t launch_tree_attn_umma(goose_ctx*, const __nv_bfloat16*, const __nv_bfloat16*, const __nv_bfloat16*, int64_t,
-                                  const int64_t*, const int32_t*, const int32_t*, int, int, int, float,
-                                  __nv_bfloat16*, float*, cudaStream_t) { return cudaErrorNotSupported; }
+
+namespace {
+
+constexpr int kTile = 128;                      // keys per tile
+constexpr int kStages = 4;                      // ring of K/V stages
+constexpr int kStageBytes = kTile * kHeadDim * 2;   // 32 KB: one K or one V tile
+constexpr int kHalfBytes = kTile * 128;         // 16 KB: 128 rows x 64 bf16 (one swizzle-atom column)
+constexpr int kQBytes = 2 * kHalfBytes;
+constexpr int kPBytes = 2 * kHalfBytes;
+constexpr int kHeaderBytes = 1024;
+constexpr int kUmmaSmem = kHeaderBytes + 1024 /*alignment slack*/ + kQBytes + kPBytes + kStages * kStageBytes;
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColS = 0, kColO = 256;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kRescaleThreshold = 8.0f;       // rescale O only when the running max grew by > 2^8
+constexpr long long kWaitCycles = 2000000000ll;  // bound of every wait: about one second of SM clock
+
+struct Header {                                  // lives at the start of dynamic shared memory
+    unsigned long long kv_full[kStages];
+    unsigned long long kv_empty[kStages];
+    unsigned long long q_full, q_empty;
+    unsigned long long s_full[2];
+    unsigned long long p_ready, pv_done, o_free;
+    unsigned long long group_bar;                // barrier of the 128 softmax threads (bounded, unlike bar.sync)
+    uint32_t tmem_base;
+    volatile int abort_flag;
+    int bad_parent;
+    int last_flag;
+    int par[kMaxB];                              // parent[] of the current segment's sequence
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
 }
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait (about one second of SM clock).  Returns false, and raises the CTA's abort flag, when it
+// gives up; returns false at once when another role has already aborted.
+__device__ __forceinline__ bool mbar_wait(Header* hd, unsigned long long* bar, uint32_t parity, int32_t* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        if (hd->abort_flag) return false;
+        if (mbar_try_wait(bar, parity)) return true;
+        if (clock64() - t0 > kWaitCycles) break;
+    }
+    hd->abort_flag = 1;
+    atomicOr(status, GOOSE_ST_TIMEOUT);
+    return false;
+}
+// Bounded wait used only while draining after an abort (ignores the abort flag).
+__device__ __forceinline__ void mbar_drain(unsigned long long* bar, uint32_t parity) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity) && clock64() - t0 < kWaitCycles) {}
+}
+
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, unsigned long long* bar,
+                                            int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+// shared-memory matrix descriptor, 128-byte swizzle; addresses and offsets in bytes
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+    return (uint64_t)((addr >> 4) & 0x3FFF) | ((uint64_t)((lbo >> 4) & 0x3FFF) << 16) |
+           ((uint64_t)((sbo >> 4) & 0x3FFF) << 32) | (1ull << 46) /*descriptor version*/ | (2ull << 61) /*SWIZZLE_128B*/;
+}
+// instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128, A K-major, B K-major or MN-major
+__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+}
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(unsigned long long* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+#define TMEM_LD32(taddr, v, off)                                                                                      \
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                            \
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"                                          \
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"                           \
+                 : "=r"(v[off + 0]), "=r"(v[off + 1]), "=r"(v[off + 2]), "=r"(v[off + 3]), "=r"(v[off + 4]),          \
+                   "=r"(v[off + 5]), "=r"(v[off + 6]), "=r"(v[off + 7]), "=r"(v[off + 8]), "=r"(v[off + 9]),          \
+                   "=r"(v[off + 10]), "=r"(v[off + 11]), "=r"(v[off + 12]), "=r"(v[off + 13]), "=r"(v[off + 14]),     \
+                   "=r"(v[off + 15]), "=r"(v[off + 16]), "=r"(v[off + 17]), "=r"(v[off + 18]), "=r"(v[off + 19]),     \
+                   "=r"(v[off + 20]), "=r"(v[off + 21]), "=r"(v[off + 22]), "=r"(v[off + 23]), "=r"(v[off + 24]),     \
+                   "=r"(v[off + 25]), "=r"(v[off + 26]), "=r"(v[off + 27]), "=r"(v[off + 28]), "=r"(v[off + 29]),     \
+                   "=r"(v[off + 30]), "=r"(v[off + 31])                                                               \
+                 : "r"(taddr))
+#define TMEM_ST32(taddr, v, off)                                                                                      \
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "                                                     \
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"                                          \
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31};"                                  \
+                 ::"r"(v[off + 0]), "r"(v[off + 1]), "r"(v[off + 2]), "r"(v[off + 3]), "r"(v[off + 4]),               \
+                   "r"(v[off + 5]), "r"(v[off + 6]), "r"(v[off + 7]), "r"(v[off + 8]), "r"(v[off + 9]),               \
+                   "r"(v[off + 10]), "r"(v[off + 11]), "r"(v[off + 12]), "r"(v[off + 13]), "r"(v[off + 14]),          \
+                   "r"(v[off + 15]), "r"(v[off + 16]), "r"(v[off + 17]), "r"(v[off + 18]), "r"(v[off + 19]),          \
+                   "r"(v[off + 20]), "r"(v[off + 21]), "r"(v[off + 22]), "r"(v[off + 23]), "r"(v[off + 24]),          \
+                   "r"(v[off + 25]), "r"(v[off + 26]), "r"(v[off + 27]), "r"(v[off + 28]), "r"(v[off + 29]),          \
+                   "r"(v[off + 30]), "r"(v[off + 31]), "r"(taddr) : "memory")
+
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+// barrier of the 128 softmax threads; `n` counts its uses (every thread calls it the same number of times)
+__device__ __forceinline__ bool group_sync(Header* hd, uint32_t& n, int32_t* status) {
+    mbar_arrive(&hd->group_bar);
+    bool ok = mbar_wait(hd, &hd->group_bar, n & 1, status);
+    ++n;
+    return ok;
+}
+
+// ---------------------------------------------------------------- work partition (same code in every role)
+struct Work {
+    const int32_t* ctx_len;
+    int S, H, B, G;
+    long long total;          // all items
+    __device__ __forceinline__ int tiles(int s) const { return (ctx_len[s] + B + kTile - 1) / kTile; }
+    __device__ __forceinline__ long long cta_start(int c) const { return total * c / G; }
+    __device__ __forceinline__ int cta_of(long long w) const {
+        int c = (int)(w * G / total);
+        if (c >= G) c = G - 1;
+        while (c + 1 < G && cta_start(c + 1) <= w) ++c;
+        while (c > 0 && cta_start(c) > w) --c;
+        return c;
+    }
+};
+
+struct Cursor {               // walks items in order
+    long long w;              // item index
+    int s, h, t, T;
+    __device__ __forceinline__ void seek(const Work& wk, long long w0) {
+        long long off = 0;
+        int ss = 0;
+        int TT = wk.tiles(0);
+        while (ss + 1 < wk.S && off + (long long)wk.H * TT <= w0) {
+            off += (long long)wk.H * TT;
+            ++ss;
+            TT = wk.tiles(ss);
+        }
+        s = ss; T = TT; w = w0;
+        h = (int)((w0 - off) / TT);
+        t = (int)((w0 - off) % TT);
+    }
+    __device__ __forceinline__ void next(const Work& wk) {
+        ++w; ++t;
+        if (t == T) {
+            t = 0; ++h;
+            if (h == wk.H) { h = 0; ++s; if (s < wk.S) T = wk.tiles(s); }
+        }
+    }
+};
+
+// ---------------------------------------------------------------- the kernel
+__global__ void __launch_bounds__(kThreads, 1)
+tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                      const __grid_constant__ CUtensorMap tmap_v, const int64_t* __restrict__ row_off,
+                      const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ parent,
+                      int S, int B, int H, float scale_log2, float* __restrict__ partials,
+                      int32_t* __restrict__ head_counters, int32_t* __restrict__ status,
+                      __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+    extern __shared__ unsigned char smem_raw[];
+    Header* hd = reinterpret_cast<Header*>(smem_raw);
+    unsigned char* buf = reinterpret_cast<unsigned char*>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + kHeaderBytes + 1023) & ~(uintptr_t)1023);
+    unsigned char* q_smem = buf;
+    unsigned char* p_smem = buf + kQBytes;
+    unsigned char* kv_smem = buf + kQBytes + kPBytes;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    Work wk;
+    wk.ctx_len = ctx_len; wk.S = S; wk.H = H; wk.B = B; wk.G = gridDim.x;
+    {
+        long long tot = 0;
+        for (int s = 0; s < S; ++s) tot += (long long)H * wk.tiles(s);
+        wk.total = tot;
+    }
+    const long long w_begin = wk.cta_start(blockIdx.x), w_end = wk.cta_start(blockIdx.x + 1);
+
+    // ---- set-up
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kStages; ++i) { mbar_init(&hd->kv_full[i], 1); mbar_init(&hd->kv_empty[i], 1); }
+        mbar_init(&hd->q_full, 1); mbar_init(&hd->q_empty, 1);
+        mbar_init(&hd->s_full[0], 1); mbar_init(&hd->s_full[1], 1);
+        mbar_init(&hd->p_ready, 128); mbar_init(&hd->pv_done, 1); mbar_init(&hd->o_free, 128);
+        mbar_init(&hd->group_bar, 128);
+        hd->abort_flag = 0; hd->bad_parent = 0; hd->last_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {                                   // TMEM: the whole 512 columns (one CTA per SM)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&hd->tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = hd->tmem_base;
+
+    if (w_begin < w_end) {
+        if (warp == 0) {
+            // =========================================================== TMA producer
+            if (lane == 0) {
+                prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
+                Cursor cu; cu.seek(wk, w_begin);
+                uint32_t ring = 0, seg = 0;
+                bool ok = true;
+                while (ok && cu.w < w_end) {
+                    const int64_t row0 = row_off[cu.s];
+                    // Q of this segment
+                    ok = mbar_wait(hd, &hd->q_empty, (seg & 1) ^ 1, status);   // seg = index of this segment
+                    if (!ok) break;
+                    mbar_expect_tx(&hd->q_full, (uint32_t)B * 256u);
+                    tma_load_3d(q_smem, &tmap_q, &hd->q_full, 0, cu.h, cu.s * B);
+                    tma_load_3d(q_smem + kHalfBytes, &tmap_q, &hd->q_full, 64, cu.h, cu.s * B);
+                    ++seg;                                 // segments whose Q load has been issued
+                    const int s0 = cu.s, h0 = cu.h;
+                    while (ok && cu.w < w_end && cu.s == s0 && cu.h == h0) {
+                        const int krow = (int)(row0 + (int64_t)cu.t * kTile);
+                        for (int kv = 0; kv < 2 && ok; ++kv) {
+                            const uint32_t st = ring % kStages, fill = ring / kStages;
+                            ok = mbar_wait(hd, &hd->kv_empty[st], (fill & 1) ^ 1, status);
+                            if (!ok) break;
+                            unsigned char* dst = kv_smem + st * kStageBytes;
+                            mbar_expect_tx(&hd->kv_full[st], kStageBytes);
+                            const CUtensorMap* mp = kv ? &tmap_v : &tmap_k;
+                            tma_load_3d(dst, mp, &hd->kv_full[st], 0, cu.h, krow);
+                            tma_load_3d(dst + kHalfBytes, mp, &hd->kv_full[st], 64, cu.h, krow);
+                            ++ring;
+                        }
+                        cu.next(wk);
+                    }
+                }
+                if (!ok) {
+                    // aborted: drain this thread's copies still in flight (bounded) before the CTA exits
+                    uint32_t first = ring > kStages ? ring - kStages : 0;
+                    for (uint32_t r = first; r < ring; ++r) mbar_drain(&hd->kv_full[r % kStages], (r / kStages) & 1);
+                    if (seg > 0) mbar_drain(&hd->q_full, (seg - 1) & 1);
+                }
+            }
+        } else if (warp == 1) {
+            // =========================================================== MMA issuer
+            if (lane == 0) {
+                Cursor cu; cu.seek(wk, w_begin);
+                uint32_t jg = 0, seg = 0;                  // CTA-global tile and segment counters
+                bool ok = true;
+                const uint32_t q_addr = smem_u32(q_smem), p_addr = smem_u32(p_smem), kv_addr = smem_u32(kv_smem);
+                constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
+
+                auto issue_pv = [&](uint32_t j, bool first_of_segment) -> bool {
+                    // tile j's P is in shared memory and S(j) has been consumed
+                    if (!mbar_wait(hd, &hd->p_ready, j & 1, status)) return false;
+                    const uint32_t ring = 2 * j + 1, st = ring % kStages;
+                    if (!mbar_wait(hd, &hd->kv_full[st], (ring / kStages) & 1, status)) return false;
+                    if (first_of_segment && seg > 0)       // the previous segment's O must have left TMEM
+                        if (!mbar_wait(hd, &hd->o_free, (seg - 1) & 1, status)) return false;
+                    tc_fence_after();
+                    const uint32_t v_addr = kv_addr + st * kStageBytes;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {       // 16 keys per instruction
+                        uint64_t a = smem_desc(p_addr + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16, 1024);
+                        uint64_t b = smem_desc(v_addr + kk * 2048, kHalfBytes, 1024);   // MN-major: LBO = next 64 d
+                        umma_f16(tmem + kColO, a, b, idesc_pv, (!first_of_segment || kk > 0) ? 1u : 0u);
+                    }
+                    umma_commit(&hd->kv_empty[st]);
+                    umma_commit(&hd->pv_done);
+                    return true;
+                };
+
+                while (ok && cu.w < w_end) {
+                    ok = mbar_wait(hd, &hd->q_full, seg & 1, status);
+                    if (!ok) break;
+                    const int s0 = cu.s, h0 = cu.h;
+                    const uint32_t j_first = jg;
+                    while (ok && cu.w < w_end && cu.s == s0 && cu.h == h0) {
+                        const uint32_t ring = 2 * jg, st = ring % kStages;
+                        ok = mbar_wait(hd, &hd->kv_full[st], (ring / kStages) & 1, status);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t k_addr = kv_addr + st * kStageBytes;
+                        const uint32_t d_tmem = tmem + kColS + (jg & 1) * 128;
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {   // 16 of the 128 head dims per instruction
+                            uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+                            umma_f16(d_tmem, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024),
+                                     idesc_qk, kk > 0 ? 1u : 0u);
+                        }
+                        umma_commit(&hd->s_full[jg & 1]);
+                        umma_commit(&hd->kv_empty[st]);
+                        if (jg > j_first) ok = issue_pv(jg - 1, jg - 1 == j_first);
+                        ++jg;
+                        cu.next(wk);
+                    }
+                    if (!ok) break;
+                    umma_commit(&hd->q_empty);             // every QK^T of the segment has been issued
+                    ok = issue_pv(jg - 1, jg - 1 == j_first);
+                    ++seg;
+                }
+            }
+        } else {
+            // =========================================================== softmax / epilogue (128 threads)
+            const int row = 32 * (warp & 3) + lane;        // TMEM lane == query row
+            const uint32_t lane_sel = (uint32_t)(32 * (warp & 3)) << 16;
+            const bool warp_has_rows = 32 * (warp & 3) < B;
+            const int sm_tid = threadIdx.x - 64;           // 0..127
+            Cursor cu; cu.seek(wk, w_begin);
+            uint32_t jg = 0, seg = 0, gsync = 0;
+            bool ok = true;
+            uint32_t v[128];
+
+            while (ok && cu.w < w_end) {
+                const int s0 = cu.s, h0 = cu.h, T = cu.T;
+                const int ctx = ctx_len[s0];
+                const int n_keys = ctx + B;
+                const int32_t* par = parent + (size_t)s0 * B;
+                const int t_first = cu.t;
+                // validate parent[] of this sequence (all 128 threads reach the same verdict)
+                if (row < B) {
+                    int p = par[row];
+                    hd->par[row] = p;
+                    if ((row == 0) ? (p != -1) : (p < 0 || p >= row)) hd->bad_parent = 1;
+                }
+                ok = group_sync(hd, gsync, status);
+                const bool bad = hd->bad_parent != 0;
+                ok = ok && group_sync(hd, gsync, status);
+                if (!ok) break;
+                if (sm_tid == 0 && bad) { hd->bad_parent = 0; atomicOr(&status[s0], GOOSE_ST_BAD_PARENT); }
+                uint32_t anc[4] = {0, 0, 0, 0};
+                if (row < B) {
+                    if (bad) {
+                        anc[row >> 5] = 1u << (row & 31);
+                    } else {
+                        int vtx = row;
+                        for (int step = 0; step < B && vtx >= 0; ++step) {
+                            uint32_t bit = 1u << (vtx & 31);
+                            int wsel = vtx >> 5;
+                            anc[0] |= (wsel == 0) ? bit : 0; anc[1] |= (wsel == 1) ? bit : 0;
+                            anc[2] |= (wsel == 2) ? bit : 0; anc[3] |= (wsel == 3) ? bit : 0;
+                            vtx = hd->par[vtx];
+                        }
+                    }
+                }
+                float m_run = -INFINITY, l_run = 0.f;
+                int seg_tiles = 0;
+
+                while (ok && cu.w < w_end && cu.s == s0 && cu.h == h0) {
+                    const int t = cu.t;
+                    const bool first = (t == t_first);
+                    ok = mbar_wait(hd, &hd->s_full[jg & 1], (jg >> 1) & 1, status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    float m_use = 0.f;
+                    if (warp_has_rows) {
+                        const uint32_t s_addr = tmem + kColS + (jg & 1) * 128 + lane_sel;
+                        TMEM_LD32(s_addr, v, 0); TMEM_LD32(s_addr + 32, v, 32);
+                        TMEM_LD32(s_addr + 64, v, 64); TMEM_LD32(s_addr + 96, v, 96);
+                        tmem_wait_ld();
+                        const int key0 = t * kTile;
+                        if (key0 + kTile > ctx) {          // this tile reaches the tree rows (or the ragged end)
+#pragma unroll
+                            for (int c = 0; c < 128; ++c) {
+                                int kk = key0 + c;
+                                bool vis = kk < ctx;
+                                if (!vis && kk < n_keys) {
+                                    int j = kk - ctx;
+                                    uint32_t wsel = (j < 32) ? anc[0] : (j < 64) ? anc[1] : (j < 96) ? anc[2] : anc[3];
+                                    vis = (wsel >> (j & 31)) & 1u;
+                                }
+                                v[c] = vis ? v[c] : 0xFF800000u;   // -inf
+                            }
+                        }
+                        float mx = -INFINITY;
+#pragma unroll
+                        for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(v[c]));
+                        mx *= scale_log2;                  // scale > 0
+                        const float m_new = fmaxf(m_run, mx);
+                        // lazy rescaling: keep the stale maximum unless it grew by more than the threshold
+                        const bool need = first ? true : (m_new > m_run + kRescaleThreshold);
+                        if (__any_sync(0xFFFFFFFFu, need)) {
+                            const float alpha = (m_run == -INFINITY) ? 0.f : ex2(m_run - m_new);
+                            if (!first) {
+                                // O holds tiles < t of this segment: wait for PV(t-1), then scale the row
+                                ok = mbar_wait(hd, &hd->pv_done, (jg - 1) & 1, status);
+                                if (ok) {
+                                    tc_fence_after();
+                                    uint32_t o[32];
+                                    const uint32_t o_addr = tmem + kColO + lane_sel;
+#pragma unroll
+                                    for (int cc = 0; cc < 4; ++cc) {
+                                        TMEM_LD32(o_addr + cc * 32, o, 0);
+                                        tmem_wait_ld();
+#pragma unroll
+                                        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                                        TMEM_ST32(o_addr + cc * 32, o, 0);
+                                    }
+                                    tmem_wait_st();
+                                }
+                            }
+                            l_run *= alpha;
+                            m_run = m_new;
+                        }
+                        m_use = (m_run == -INFINITY) ? 0.f : m_run;
+                    }
+                    // P(jg) may overwrite P(jg-1) only after PV(jg-1) has read it
+                    if (ok && jg > 0) ok = mbar_wait(hd, &hd->pv_done, (jg - 1) & 1, status);
+                    if (!ok) break;
+                    if (warp_has_rows) {
+                        float lsum = 0.f;
+                        const float neg_m = -m_use;
+                        unsigned char* prow = p_smem + row * 128;
+#pragma unroll
+                        for (int ch = 0; ch < 16; ++ch) {  // 16-byte chunks of 8 keys
+                            uint32_t pk[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                float p0 = ex2(fmaf(__uint_as_float(v[ch * 8 + 2 * e]), scale_log2, neg_m));
+                                float p1 = ex2(fmaf(__uint_as_float(v[ch * 8 + 2 * e + 1]), scale_log2, neg_m));
+                                lsum += p0 + p1;
+                                pk[e] = pack_bf16x2(p0, p1);
+                            }
+                            const int half = ch >> 3, cin = ch & 7;
+                            *reinterpret_cast<uint4*>(prow + half * kHalfBytes + ((cin ^ (row & 7)) << 4)) =
+                                make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        }
+                        l_run += lsum;
+                    }
+                    // ragged end: V rows past the sequence's last key may hold anything -> zero them
+                    if ((t + 1) * kTile > n_keys) {
+                        const uint32_t ring = 2 * jg + 1, st = ring % kStages;
+                        ok = mbar_wait(hd, &hd->kv_full[st], (ring / kStages) & 1, status);
+                        if (!ok) break;
+                        const int r_local = sm_tid;        // one V row (key) per thread
+                        if (t * kTile + r_local >= n_keys) {
+                            unsigned char* vrow = kv_smem + st * kStageBytes + r_local * 128;
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) {
+                                *reinterpret_cast<uint4*>(vrow + c * 16) = make_uint4(0, 0, 0, 0);
+                                *reinterpret_cast<uint4*>(vrow + kHalfBytes + c * 16) = make_uint4(0, 0, 0, 0);
+                            }
+                        }
+                    }
+                    fence_proxy_async();                   // generic-proxy writes -> visible to the tensor core
+                    tc_fence_before();
+                    mbar_arrive(&hd->p_ready);
+                    ++jg;
+                    ++seg_tiles;
+                    cu.next(wk);
+                }
+                if (!ok) break;
+
+                // ---------------- segment epilogue: O of tiles [t_first, t_last] is complete after PV(jg-1)
+                ok = mbar_wait(hd, &hd->pv_done, (jg - 1) & 1, status);
+                if (!ok) break;
+                tc_fence_after();
+                const int n_tiles_seg = seg_tiles;
+                const bool whole_head = (t_first == 0) && (n_tiles_seg == T);
+                if (warp_has_rows) {
+                    const uint32_t o_addr = tmem + kColO + lane_sel;
+                    TMEM_LD32(o_addr, v, 0); TMEM_LD32(o_addr + 32, v, 32);
+                    TMEM_LD32(o_addr + 64, v, 64); TMEM_LD32(o_addr + 96, v, 96);
+                    tmem_wait_ld();
+                }
+                tc_fence_before();
+                mbar_arrive(&hd->o_free);                  // TMEM O may be overwritten by the next segment
+
+                const size_t head = (size_t)s0 * H + h0;
+                if (whole_head) {
+                    if (row < B) {
+                        const float inv = bad ? 0.f : 1.f / l_run;
+                        uint4* dst = reinterpret_cast<uint4*>(out + (((size_t)s0 * B + row) * H + h0) * kHeadDim);
+#pragma unroll
+                        for (int ch = 0; ch < 16; ++ch) {
+                            uint32_t pk[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                pk[e] = bad ? 0u : pack_bf16x2(__uint_as_float(v[ch * 8 + 2 * e]) * inv,
+                                                               __uint_as_float(v[ch * 8 + 2 * e + 1]) * inv);
+                            dst[ch] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        }
+                        if (lse) lse[((size_t)s0 * B + row) * H + h0] = bad ? 0.f : (m_run + log2f(l_run)) * kLn2;
+                    }
+                } else {
+                    // partial -> workspace; the last CTA to arrive for this head combines
+                    const int slot = 2 * blockIdx.x + (t_first == 0 ? 1 : 0);
+                    float* part = partials + (size_t)slot * kPartialFloats;
+                    if (row < B) {
+                        float4* dst = reinterpret_cast<float4*>(part + row * kHeadDim);
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            dst[c] = make_float4(__uint_as_float(v[4 * c]), __uint_as_float(v[4 * c + 1]),
+                                                 __uint_as_float(v[4 * c + 2]), __uint_as_float(v[4 * c + 3]));
+                        part[kMaxB * kHeadDim + row] = m_run;
+                        part[kMaxB * kHeadDim + kMaxB + row] = l_run;
+                    }
+                    __threadfence();
+                    ok = group_sync(hd, gsync, status);
+                    if (!ok) break;
+                    // first item of this head: the segment started at item w_seg0 with tile t_first
+                    const long long w_seg0 = cu.w - n_tiles_seg;
+                    const long long head_first = w_seg0 - t_first;
+                    const int c_lo = wk.cta_of(head_first), c_hi = wk.cta_of(head_first + T - 1);
+                    const int nparts = c_hi - c_lo + 1;
+                    if (sm_tid == 0) {
+                        int old = atomicAdd(&head_counters[head], 1);
+                        hd->last_flag = (old == nparts - 1);
+                        if (old == nparts - 1) head_counters[head] = 0;   // ready for the next launch
+                    }
+                    ok = group_sync(hd, gsync, status);
+                    const bool last = hd->last_flag != 0;
+                    ok = ok && group_sync(hd, gsync, status);
+                    if (!ok) break;
+                    if (last) {
+                        __threadfence();
+                        // thread d handles output column d of every row (coalesced reads of the partials)
+                        const int d = sm_tid;
+                        for (int i = 0; i < B; ++i) {
+                            float M = -INFINITY;
+                            for (int c = c_lo; c <= c_hi; ++c) {
+                                const long long cs = wk.cta_start(c);
+                                const int sl = 2 * c + ((cs <= head_first) ? 1 : 0);
+                                M = fmaxf(M, __ldcg(partials + (size_t)sl * kPartialFloats + kMaxB * kHeadDim + i));
+                            }
+                            float L = 0.f, acc = 0.f;
+                            for (int c = c_lo; c <= c_hi; ++c) {
+                                const long long cs = wk.cta_start(c);
+                                const int sl = 2 * c + ((cs <= head_first) ? 1 : 0);
+                                const float* pp = partials + (size_t)sl * kPartialFloats;
+                                const float mp = __ldcg(pp + kMaxB * kHeadDim + i);
+                                const float wgt = (mp == -INFINITY) ? 0.f : ex2(mp - M);
+                                L += wgt * __ldcg(pp + kMaxB * kHeadDim + kMaxB + i);
+                                acc += wgt * __ldcg(pp + i * kHeadDim + d);
+                            }
+                            const float r = bad ? 0.f : acc / L;
+                            out[(((size_t)s0 * B + i) * H + h0) * kHeadDim + d] = __float2bfloat16_rn(r);
+                            if (lse && d == 0) lse[((size_t)s0 * B + i) * H + h0] = bad ? 0.f : (M + log2f(L)) * kLn2;
+                        }
+                    }
+                }
+                ++seg;
+            }
+        }
+    }
+
+    // ---- teardown
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// bf16 tensor [rows][H][128] -> 3-D map, box = 64 x 1 x box_rows, 128-byte swizzle, zero fill out of bounds
+bool make_map(void* fn, CUtensorMap* map, const void* base, int64_t rows, int H, int box_rows) {
+    cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)H, (cuuint64_t)rows};
+    cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)H * kHeadDim * 2};
+    cuuint32_t box[3] = {64, 1, (cuuint32_t)box_rows};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = reinterpret_cast<EncodeTiledFn>(fn)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base),
+                                                     dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+cudaError_t init_umma_kernel() {
+    return cudaFuncSetAttribute(tree_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmem);
+}
+
+int auto_attn_impl(const goose_ctx* c, int S, int B, int H) {
+    (void)S; (void)H;
+    if (!c->encode_tiled) return GOOSE_ATTN_MMA;
+    return B >= 32 ? GOOSE_ATTN_UMMA : GOOSE_ATTN_MMA;
+}
+
+cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __nv_bfloat16* kc,
+                                  const __nv_bfloat16* vc, int64_t kv_rows, const int64_t* row_off,
+                                  const int32_t* ctx_len, const int32_t* parent, int S, int B, int H,
+                                  float scale, __nv_bfloat16* out, float* lse, cudaStream_t st) {
+    if (!c->encode_tiled) return cudaErrorNotSupported;
+    if (S == 0) return cudaSuccess;
+    CUtensorMap mq, mk, mv;
+    if (!make_map(c->encode_tiled, &mq, q, (int64_t)S * B, H, B) ||
+        !make_map(c->encode_tiled, &mk, kc, kv_rows, H, kTile) ||
+        !make_map(c->encode_tiled, &mv, vc, kv_rows, H, kTile))
+        return cudaErrorInvalidValue;
+    int grid = c->num_sms;
+    if (2 * grid > c->n_slots) grid = c->n_slots / 2;
+    tree_attn_umma_kernel<<<grid, kThreads, kUmmaSmem, st>>>(mq, mk, mv, row_off, ctx_len, parent, S, B, H,
+                                                            scale * kLog2e, c->partials, c->head_counters, c->status,
+                                                            out, lse);
+    c->launches++;
+    return cudaGetLastError();
+}
+
+}  // namespace goose

@@ -563,7 +563,8 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                     const long long w_seg0 = cu.w - n_tiles_seg;
                     const long long head_first = w_seg0 - t_first;
                     const int c_lo = wk.cta_of(head_first), c_hi = wk.cta_of(head_first + T - 1);
-                    const int nparts = c_hi - c_lo + 1;
+                    int nparts = 0;                        // CTAs with a non-empty share of this head
+                    for (int c = c_lo; c <= c_hi; ++c) nparts += wk.cta_start(c + 1) > wk.cta_start(c);
                     if (sm_tid == 0) {
                         int old = atomicAdd(&head_counters[head], 1);
                         hd->last_flag = (old == nparts - 1);
@@ -581,12 +582,14 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                             float M = -INFINITY;
                             for (int c = c_lo; c <= c_hi; ++c) {
                                 const long long cs = wk.cta_start(c);
+                                if (wk.cta_start(c + 1) == cs) continue;
                                 const int sl = 2 * c + ((cs <= head_first) ? 1 : 0);
                                 M = fmaxf(M, __ldcg(partials + (size_t)sl * kPartialFloats + kMaxB * kHeadDim + i));
                             }
                             float L = 0.f, acc = 0.f;
                             for (int c = c_lo; c <= c_hi; ++c) {
                                 const long long cs = wk.cta_start(c);
+                                if (wk.cta_start(c + 1) == cs) continue;
                                 const int sl = 2 * c + ((cs <= head_first) ? 1 : 0);
                                 const float* pp = partials + (size_t)sl * kPartialFloats;
                                 const float mp = __ldcg(pp + kMaxB * kHeadDim + i);

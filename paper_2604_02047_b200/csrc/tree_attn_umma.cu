@@ -5,8 +5,8 @@
 // (one per SM) in contiguous ranges, so every SM streams the same number of K/V bytes.  A run of
 // items of one head inside a CTA's range is a "segment"; a segment that covers its whole head
 // writes the bf16 output directly, any other segment writes an fp32 partial (unnormalised O, running
-// max m, running sum l) and the last CTA to arrive for the head (arrival counter, no spinning)
-// combines the partials.
+// max m, running sum l) to the workspace, and a small second kernel (tree_attn_combine_kernel, spread
+// over all SMs) merges the partials of every head that was split.
 //
 // Roles (192 threads):
 //   warp 0, lane 0   TMA producer: Q of the segment, then K and V tiles into a ring of 32 KB stages
@@ -14,7 +14,7 @@
 //   warps 2..5       softmax:      one query row per thread (TMEM lane = row): S from TMEM, ancestor
 //                                  mask on the tiles that reach the tree rows, exp2, P (bf16) into
 //                                  shared memory in the canonical 128-byte-swizzled K-major layout,
-//                                  lazy rescaling of O in TMEM, epilogue / partial / combine.
+//                                  lazy rescaling of O in TMEM, epilogue (output or partial).
 // All B <= 128 query rows ride in one M = 128 MMA; rows >= B compute on don't-care data and are
 // never written out.  The tree part of the mask (Sec. 4 Stage 1: a node attends to the prefix and to
 // its root-to-node ancestors) is a per-row 128-bit ancestor set built from parent[].
@@ -43,7 +43,24 @@ constexpr uint32_t kColS = 0, kColO = 256;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;       // rescale O only when the running max grew by > 2^8
+constexpr int kCombineChunk = 8;                 // partials merged per pass of the combine kernel
 constexpr long long kWaitCycles = 2000000000ll;  // bound of every wait: about one second of SM clock
+
+#ifdef GOOSE_TRACE
+// Debug build only: per-CTA, per-role timestamp log (64 entries of tag<<56 | globaltimer ns per role).
+__device__ unsigned long long* g_trace = nullptr;
+__device__ __forceinline__ void trace_ev(int role, int& n, unsigned tag) {
+    if (g_trace && n < 64) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        g_trace[((size_t)blockIdx.x * 3 + role) * 64 + n] = ((unsigned long long)tag << 56) | (t & 0x00FFFFFFFFFFFFFFull);
+        ++n;
+    }
+}
+#define TRACE(role, n, tag) trace_ev(role, n, tag)
+#else
+#define TRACE(role, n, tag) do { } while (0)
+#endif
 
 struct Header {                                  // lives at the start of dynamic shared memory
     unsigned long long kv_full[kStages];
@@ -55,7 +72,6 @@ struct Header {                                  // lives at the start of dynami
     uint32_t tmem_base;
     volatile int abort_flag;
     int bad_parent;
-    int last_flag;
     int par[kMaxB];                              // parent[] of the current segment's sequence
 };
 
@@ -105,6 +121,17 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, u
                                             int c0, int c1, int c2) {
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
                  ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_hint(void* dst, const CUtensorMap* map, unsigned long long* bar,
+                                                 int c0, int c1, int c2, unsigned long long policy) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+                 "[%0], [%1, {%3, %4, %5}], [%2], %6;"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "l"(policy) : "memory");
+}
+__device__ __forceinline__ unsigned long long l2_policy_evict_first() {
+    unsigned long long pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -220,7 +247,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                       const __grid_constant__ CUtensorMap tmap_v, const int64_t* __restrict__ row_off,
                       const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ parent,
                       int S, int B, int H, float scale_log2, float* __restrict__ partials,
-                      int32_t* __restrict__ head_counters, int32_t* __restrict__ status,
+                      int32_t* __restrict__ status,
                       __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
     extern __shared__ unsigned char smem_raw[];
     Header* hd = reinterpret_cast<Header*>(smem_raw);
@@ -248,7 +275,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
         mbar_init(&hd->s_full[0], 1); mbar_init(&hd->s_full[1], 1);
         mbar_init(&hd->p_ready, 128); mbar_init(&hd->pv_done, 1); mbar_init(&hd->o_free, 128);
         mbar_init(&hd->group_bar, 128);
-        hd->abort_flag = 0; hd->bad_parent = 0; hd->last_flag = 0;
+        hd->abort_flag = 0; hd->bad_parent = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {                                   // TMEM: the whole 512 columns (one CTA per SM)
@@ -266,9 +293,14 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
             // =========================================================== TMA producer
             if (lane == 0) {
                 prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
+                // K and V are read exactly once: mark them evict-first so that the split-KV partials
+                // (written and re-read within this launch) stay resident in L2
+                const unsigned long long pol_stream = l2_policy_evict_first();
                 Cursor cu; cu.seek(wk, w_begin);
                 uint32_t ring = 0, seg = 0;
                 bool ok = true;
+                int tn = 0; (void)tn;
+                TRACE(0, tn, 1);
                 while (ok && cu.w < w_end) {
                     const int64_t row0 = row_off[cu.s];
                     // Q of this segment
@@ -288,9 +320,10 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                             unsigned char* dst = kv_smem + st * kStageBytes;
                             mbar_expect_tx(&hd->kv_full[st], kStageBytes);
                             const CUtensorMap* mp = kv ? &tmap_v : &tmap_k;
-                            tma_load_3d(dst, mp, &hd->kv_full[st], 0, cu.h, krow);
-                            tma_load_3d(dst + kHalfBytes, mp, &hd->kv_full[st], 64, cu.h, krow);
+                            tma_load_3d_hint(dst, mp, &hd->kv_full[st], 0, cu.h, krow, pol_stream);
+                            tma_load_3d_hint(dst + kHalfBytes, mp, &hd->kv_full[st], 64, cu.h, krow, pol_stream);
                             ++ring;
+                            TRACE(0, tn, 2);
                         }
                         cu.next(wk);
                     }
@@ -308,6 +341,8 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 Cursor cu; cu.seek(wk, w_begin);
                 uint32_t jg = 0, seg = 0;                  // CTA-global tile and segment counters
                 bool ok = true;
+                int tn = 0; (void)tn;
+                TRACE(1, tn, 1);
                 const uint32_t q_addr = smem_u32(q_smem), p_addr = smem_u32(p_smem), kv_addr = smem_u32(kv_smem);
                 constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
 
@@ -328,6 +363,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                     }
                     umma_commit(&hd->kv_empty[st]);
                     umma_commit(&hd->pv_done);
+                    TRACE(1, tn, 3);
                     return true;
                 };
 
@@ -350,6 +386,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                                      idesc_qk, kk > 0 ? 1u : 0u);
                         }
                         umma_commit(&hd->s_full[jg & 1]);
+                        TRACE(1, tn, 2);
                         umma_commit(&hd->kv_empty[st]);
                         if (jg > j_first) ok = issue_pv(jg - 1, jg - 1 == j_first);
                         ++jg;
@@ -371,6 +408,8 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
             uint32_t jg = 0, seg = 0, gsync = 0;
             bool ok = true;
             uint32_t v[128];
+            int tn = 0; (void)tn;
+            if (sm_tid == 0) TRACE(2, tn, 1);
 
             while (ok && cu.w < w_end) {
                 const int s0 = cu.s, h0 = cu.h, T = cu.T;
@@ -413,6 +452,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                     ok = mbar_wait(hd, &hd->s_full[jg & 1], (jg >> 1) & 1, status);
                     if (!ok) break;
                     tc_fence_after();
+                    if (sm_tid == 0 && seg_tiles < 2) TRACE(2, tn, 2);
                     float m_use = 0.f;
                     if (warp_has_rows) {
                         const uint32_t s_addr = tmem + kColS + (jg & 1) * 128 + lane_sel;
@@ -421,17 +461,21 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                         tmem_wait_ld();
                         const int key0 = t * kTile;
                         if (key0 + kTile > ctx) {          // this tile reaches the tree rows (or the ragged end)
+                            // visibility of the tile's 128 keys as one 128-bit mask: the prefix keys
+                            // (c < ctx - key0) and the ancestor set shifted to where the tree rows start
+                            const int pc = ctx - key0;     // tile column of tree node 0 (may be < 0 or >= 128)
+                            const unsigned __int128 a128 =
+                                ((unsigned __int128)(((unsigned long long)anc[3] << 32) | anc[2]) << 64) |
+                                (unsigned __int128)(((unsigned long long)anc[1] << 32) | anc[0]);
+                            unsigned __int128 vm;
+                            if (pc >= 128) vm = ~(unsigned __int128)0;
+                            else if (pc > 0) vm = (((unsigned __int128)1 << pc) - 1) | (a128 << pc);
+                            else if (pc > -128) vm = a128 >> (-pc);
+                            else vm = 0;
+                            const uint32_t vw[4] = {(uint32_t)vm, (uint32_t)(vm >> 32), (uint32_t)(vm >> 64), (uint32_t)(vm >> 96)};
 #pragma unroll
-                            for (int c = 0; c < 128; ++c) {
-                                int kk = key0 + c;
-                                bool vis = kk < ctx;
-                                if (!vis && kk < n_keys) {
-                                    int j = kk - ctx;
-                                    uint32_t wsel = (j < 32) ? anc[0] : (j < 64) ? anc[1] : (j < 96) ? anc[2] : anc[3];
-                                    vis = (wsel >> (j & 31)) & 1u;
-                                }
-                                v[c] = vis ? v[c] : 0xFF800000u;   // -inf
-                            }
+                            for (int c = 0; c < 128; ++c)
+                                v[c] = ((vw[c >> 5] >> (c & 31)) & 1u) ? v[c] : 0xFF800000u;   // -inf
                         }
                         float mx = -INFINITY;
 #pragma unroll
@@ -506,6 +550,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                     fence_proxy_async();                   // generic-proxy writes -> visible to the tensor core
                     tc_fence_before();
                     mbar_arrive(&hd->p_ready);
+                    if (sm_tid == 0 && seg_tiles < 2) TRACE(2, tn, 3);
                     ++jg;
                     ++seg_tiles;
                     cu.next(wk);
@@ -516,6 +561,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 ok = mbar_wait(hd, &hd->pv_done, (jg - 1) & 1, status);
                 if (!ok) break;
                 tc_fence_after();
+                if (sm_tid == 0) TRACE(2, tn, 4);
                 const int n_tiles_seg = seg_tiles;
                 const bool whole_head = (t_first == 0) && (n_tiles_seg == T);
                 if (warp_has_rows) {
@@ -527,7 +573,6 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 tc_fence_before();
                 mbar_arrive(&hd->o_free);                  // TMEM O may be overwritten by the next segment
 
-                const size_t head = (size_t)s0 * H + h0;
                 if (whole_head) {
                     if (row < B) {
                         const float inv = bad ? 0.f : 1.f / l_run;
@@ -544,65 +589,23 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                         if (lse) lse[((size_t)s0 * B + row) * H + h0] = bad ? 0.f : (m_run + log2f(l_run)) * kLn2;
                     }
                 } else {
-                    // partial -> workspace; the last CTA to arrive for this head combines
+                    // partial -> workspace slot of this CTA (combined by tree_attn_combine_kernel).
+                    // Layout: float4 [32 column groups][128 rows] so that a warp's stores (and the
+                    // combine kernel's loads) are contiguous, then m[128], l[128].
                     const int slot = 2 * blockIdx.x + (t_first == 0 ? 1 : 0);
                     float* part = partials + (size_t)slot * kPartialFloats;
                     if (row < B) {
-                        float4* dst = reinterpret_cast<float4*>(part + row * kHeadDim);
+                        float4* dst = reinterpret_cast<float4*>(part) + row;
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
-                            dst[c] = make_float4(__uint_as_float(v[4 * c]), __uint_as_float(v[4 * c + 1]),
-                                                 __uint_as_float(v[4 * c + 2]), __uint_as_float(v[4 * c + 3]));
+                            dst[c * 128] = make_float4(__uint_as_float(v[4 * c]), __uint_as_float(v[4 * c + 1]),
+                                                       __uint_as_float(v[4 * c + 2]), __uint_as_float(v[4 * c + 3]));
                         part[kMaxB * kHeadDim + row] = m_run;
                         part[kMaxB * kHeadDim + kMaxB + row] = l_run;
                     }
-                    __threadfence();
-                    ok = group_sync(hd, gsync, status);
-                    if (!ok) break;
-                    // first item of this head: the segment started at item w_seg0 with tile t_first
-                    const long long w_seg0 = cu.w - n_tiles_seg;
-                    const long long head_first = w_seg0 - t_first;
-                    const int c_lo = wk.cta_of(head_first), c_hi = wk.cta_of(head_first + T - 1);
-                    int nparts = 0;                        // CTAs with a non-empty share of this head
-                    for (int c = c_lo; c <= c_hi; ++c) nparts += wk.cta_start(c + 1) > wk.cta_start(c);
-                    if (sm_tid == 0) {
-                        int old = atomicAdd(&head_counters[head], 1);
-                        hd->last_flag = (old == nparts - 1);
-                        if (old == nparts - 1) head_counters[head] = 0;   // ready for the next launch
-                    }
-                    ok = group_sync(hd, gsync, status);
-                    const bool last = hd->last_flag != 0;
-                    ok = ok && group_sync(hd, gsync, status);
-                    if (!ok) break;
-                    if (last) {
-                        __threadfence();
-                        // thread d handles output column d of every row (coalesced reads of the partials)
-                        const int d = sm_tid;
-                        for (int i = 0; i < B; ++i) {
-                            float M = -INFINITY;
-                            for (int c = c_lo; c <= c_hi; ++c) {
-                                const long long cs = wk.cta_start(c);
-                                if (wk.cta_start(c + 1) == cs) continue;
-                                const int sl = 2 * c + ((cs <= head_first) ? 1 : 0);
-                                M = fmaxf(M, __ldcg(partials + (size_t)sl * kPartialFloats + kMaxB * kHeadDim + i));
-                            }
-                            float L = 0.f, acc = 0.f;
-                            for (int c = c_lo; c <= c_hi; ++c) {
-                                const long long cs = wk.cta_start(c);
-                                if (wk.cta_start(c + 1) == cs) continue;
-                                const int sl = 2 * c + ((cs <= head_first) ? 1 : 0);
-                                const float* pp = partials + (size_t)sl * kPartialFloats;
-                                const float mp = __ldcg(pp + kMaxB * kHeadDim + i);
-                                const float wgt = (mp == -INFINITY) ? 0.f : ex2(mp - M);
-                                L += wgt * __ldcg(pp + kMaxB * kHeadDim + kMaxB + i);
-                                acc += wgt * __ldcg(pp + i * kHeadDim + d);
-                            }
-                            const float r = bad ? 0.f : acc / L;
-                            out[(((size_t)s0 * B + i) * H + h0) * kHeadDim + d] = __float2bfloat16_rn(r);
-                            if (lse && d == 0) lse[((size_t)s0 * B + i) * H + h0] = bad ? 0.f : (M + log2f(L)) * kLn2;
-                        }
-                    }
+                    if (sm_tid == 0) TRACE(2, tn, 5);
                 }
+                if (sm_tid == 0) TRACE(2, tn, 8);
                 ++seg;
             }
         }
@@ -616,6 +619,113 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
+}
+
+// ---------------------------------------------------------------- combine of the split-KV partials
+// Grid (row groups of 32, H, S), 128 threads.  A head that one CTA of the main kernel covered entirely
+// was written directly and is skipped; any other head is the merge of its CTAs' partials:
+//   M = max m_p,  L = sum l_p 2^(m_p - M),  out = sum_p 2^(m_p - M) O_p / L.
+// Lane <-> row (coalesced float4 loads of the transposed partial layout), warp <-> 32 output columns.
+__global__ void __launch_bounds__(128)
+tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ parent,
+                         int S, int B, int H, int G, const float* __restrict__ partials,
+                         __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+    __shared__ int slot_s[kCombineChunk];
+    const int rg = blockIdx.x, h = blockIdx.y, s = blockIdx.z;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    Work wk;
+    wk.ctx_len = ctx_len; wk.S = S; wk.H = H; wk.B = B; wk.G = G;
+    long long tot = 0, off = 0;
+    for (int ss = 0; ss < S; ++ss) {
+        if (ss == s) off = tot;
+        tot += (long long)H * wk.tiles(ss);
+    }
+    wk.total = tot;
+    const int T = wk.tiles(s);
+    const long long head_first = off + (long long)h * T;
+    const int c_lo = wk.cta_of(head_first), c_hi = wk.cta_of(head_first + T - 1);
+    if (c_lo == c_hi) return;                              // written directly by the main kernel
+    // invalid parent[] -> zero-filled output (the main kernel has already set the status word)
+    int bad = 0;
+    for (int i = tid; i < B; i += 128) {
+        int p = parent[(size_t)s * B + i];
+        bad |= (i == 0) ? (p != -1) : (p < 0 || p >= i);
+    }
+    bad = __syncthreads_or(bad);
+    const int row = rg * 32 + lane;
+    const bool row_ok = row < B;
+    float M_run = -INFINITY, L_run = 0.f;
+    float4 acc[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+    // parts in chunks; a running (M, L) with rescaling of the accumulators keeps chunks independent
+    for (int cb = c_lo; cb <= c_hi; cb += kCombineChunk) {
+        __syncthreads();
+        if (tid < kCombineChunk) {
+            const int c = cb + tid;
+            int sl = -1;
+            if (c <= c_hi) {
+                const long long cs = wk.cta_start(c);
+                if (wk.cta_start(c + 1) > cs) sl = 2 * c + ((cs <= head_first) ? 1 : 0);
+            }
+            slot_s[tid] = sl;
+        }
+        __syncthreads();
+        // this chunk's row statistics (every warp computes them for its own lanes' rows)
+        float mp[kCombineChunk], lp[kCombineChunk];
+#pragma unroll
+        for (int pi = 0; pi < kCombineChunk; ++pi) {
+            const int sl = slot_s[pi];
+            const float* pp = partials + (size_t)(sl < 0 ? 0 : sl) * kPartialFloats + kMaxB * kHeadDim;
+            const bool use = sl >= 0 && row_ok;
+            mp[pi] = use ? __ldcg(pp + row) : -INFINITY;
+            lp[pi] = use ? __ldcg(pp + kMaxB + row) : 0.f;
+        }
+        float M_new = M_run;
+#pragma unroll
+        for (int pi = 0; pi < kCombineChunk; ++pi) M_new = fmaxf(M_new, mp[pi]);
+        const float a_old = (M_run == -INFINITY) ? 0.f : ex2(M_run - M_new);
+        L_run *= a_old;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { acc[u].x *= a_old; acc[u].y *= a_old; acc[u].z *= a_old; acc[u].w *= a_old; }
+#pragma unroll
+        for (int pi = 0; pi < kCombineChunk; ++pi) {
+            const float w = (mp[pi] == -INFINITY) ? 0.f : ex2(mp[pi] - M_new);
+            L_run += w * lp[pi];
+            mp[pi] = w;                                    // reuse as the part's weight for this row
+        }
+        M_run = M_new;
+        // accumulate: warp w owns column groups 8w .. 8w+7 (32 output columns)
+#pragma unroll
+        for (int pi = 0; pi < kCombineChunk; pi += 2) {
+            const int sl0 = slot_s[pi], sl1 = slot_s[pi + 1];
+            if (sl0 < 0 && sl1 < 0) continue;             // uniform over the CTA
+            const float4* p0 = reinterpret_cast<const float4*>(partials + (size_t)(sl0 < 0 ? 0 : sl0) * kPartialFloats) + (row_ok ? row : 0);
+            const float4* p1 = reinterpret_cast<const float4*>(partials + (size_t)(sl1 < 0 ? 0 : sl1) * kPartialFloats) + (row_ok ? row : 0);
+            float4 x0[8], x1[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                x0[u] = __ldcg(p0 + (8 * warp + u) * 128);
+                x1[u] = __ldcg(p1 + (8 * warp + u) * 128);
+            }
+            const float w0 = sl0 < 0 ? 0.f : mp[pi], w1 = sl1 < 0 ? 0.f : mp[pi + 1];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                acc[u].x += w0 * x0[u].x + w1 * x1[u].x; acc[u].y += w0 * x0[u].y + w1 * x1[u].y;
+                acc[u].z += w0 * x0[u].z + w1 * x1[u].z; acc[u].w += w0 * x0[u].w + w1 * x1[u].w;
+            }
+        }
+    }
+    if (!row_ok) return;
+    const float inv = bad ? 0.f : 1.f / L_run;
+    uint4* dst = reinterpret_cast<uint4*>(out + (((size_t)s * B + row) * H + h) * kHeadDim + 32 * warp);
+#pragma unroll
+    for (int u = 0; u < 8; u += 2)
+        dst[u >> 1] = make_uint4(pack_bf16x2(acc[u].x * inv, acc[u].y * inv), pack_bf16x2(acc[u].z * inv, acc[u].w * inv),
+                                 pack_bf16x2(acc[u + 1].x * inv, acc[u + 1].y * inv),
+                                 pack_bf16x2(acc[u + 1].z * inv, acc[u + 1].w * inv));
+    if (lse && warp == 0) lse[((size_t)s * B + row) * H + h] = bad ? 0.f : (M_run + log2f(L_run)) * kLn2;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -636,6 +746,13 @@ bool make_map(void* fn, CUtensorMap* map, const void* base, int64_t rows, int H,
 }
 
 }  // namespace
+
+#ifdef GOOSE_TRACE
+extern "C" int goose_debug_set_trace(void* dev_ptr) {
+    unsigned long long* p = static_cast<unsigned long long*>(dev_ptr);
+    return (int)cudaMemcpyToSymbol(g_trace, &p, sizeof p);
+}
+#endif
 
 cudaError_t init_umma_kernel() {
     return cudaFuncSetAttribute(tree_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmem);
@@ -661,8 +778,13 @@ cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __
     int grid = c->num_sms;
     if (2 * grid > c->n_slots) grid = c->n_slots / 2;
     tree_attn_umma_kernel<<<grid, kThreads, kUmmaSmem, st>>>(mq, mk, mv, row_off, ctx_len, parent, S, B, H,
-                                                            scale * kLog2e, c->partials, c->head_counters, c->status,
+                                                            scale * kLog2e, c->partials, c->status,
                                                             out, lse);
+    c->launches++;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    dim3 cgrid((B + 31) / 32, H, S);
+    tree_attn_combine_kernel<<<cgrid, 128, 0, st>>>(ctx_len, parent, S, B, H, grid, c->partials, out, lse);
     c->launches++;
     return cudaGetLastError();
 }

@@ -280,22 +280,24 @@ def run_ours(args, x, cfg, rank, world, local_rank):
     h2d = sum(t.numel() * t.element_size() for t in hin.values()) + 2 * k_new.numel() * 2
     d2h = sum(t.numel() * t.element_size() for t in houts.values())
     e2e_steps = max(3, min(args.steps, 50))
-    with torch.cuda.stream(stream):
-        def host_step(i):
-            d = reps[i % R]
-            g.verify_step_host(d["k_cache"], d["v_cache"], hin["q"], k_new, v_new, hin["row_off"], hin["ctx_len"],
-                               hin["parent"], hin["draft_tok"], hin["logits"], x.k, x.scale, houts)
-        for i in range(3):
-            host_step(i)
-        torch.cuda.synchronize(dev)
-        dist_barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for i in range(e2e_steps):
-            host_step(i)
-        e1.record(stream)
-        torch.cuda.synchronize(dev)
-        e2e_ms = e0.elapsed_time(e1)
+    e2e_ms = float("nan")
+    if not args.no_e2e:
+        with torch.cuda.stream(stream):
+            def host_step(i):
+                d = reps[i % R]
+                g.verify_step_host(d["k_cache"], d["v_cache"], hin["q"], k_new, v_new, hin["row_off"],
+                                   hin["ctx_len"], hin["parent"], hin["draft_tok"], hin["logits"], x.k, x.scale, houts)
+            for i in range(3):
+                host_step(i)
+            torch.cuda.synchronize(dev)
+            dist_barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for i in range(e2e_steps):
+                host_step(i)
+            e1.record(stream)
+            torch.cuda.synchronize(dev)
+            e2e_ms = e0.elapsed_time(e1)
     e2e_value, _ = aggregate_steps_per_s(e2e_steps, e2e_ms, world, dev)
 
     status = g.last_status(x.S)
@@ -345,6 +347,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--attn-impl", choices=["mma", "umma"], default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 

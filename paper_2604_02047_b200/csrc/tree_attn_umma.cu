@@ -36,7 +36,7 @@ constexpr int kHalfBytes = kTile * 128;         // 16 KB: 128 rows x 64 bf16 (on
 constexpr int kQBytes = 2 * kHalfBytes;
 constexpr int kPBytes = 2 * kHalfBytes;
 constexpr int kHeaderBytes = 1024;
-constexpr int kUmmaSmem = kHeaderBytes + 1024 /*alignment slack*/ + kQBytes + kPBytes + kStages * kStageBytes;
+constexpr int kUmmaSmem = kHeaderBytes + 1024 /*alignment slack*/ + 2 * kQBytes + kPBytes + kStages * kStageBytes;
 constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;
@@ -65,7 +65,7 @@ __device__ __forceinline__ void trace_ev(int role, int& n, unsigned tag) {
 struct Header {                                  // lives at the start of dynamic shared memory
     unsigned long long kv_full[kStages];
     unsigned long long kv_empty[kStages];
-    unsigned long long q_full, q_empty;
+    unsigned long long q_full[2], q_empty[2];    // Q is double buffered: the next segment's Q is prefetched
     unsigned long long s_full[2];
     unsigned long long p_ready, pv_done, o_free;
     unsigned long long group_bar;                // barrier of the 128 softmax threads (bounded, unlike bar.sync)
@@ -254,8 +254,8 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     unsigned char* buf = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + kHeaderBytes + 1023) & ~(uintptr_t)1023);
     unsigned char* q_smem = buf;
-    unsigned char* p_smem = buf + kQBytes;
-    unsigned char* kv_smem = buf + kQBytes + kPBytes;
+    unsigned char* p_smem = buf + 2 * kQBytes;
+    unsigned char* kv_smem = buf + 2 * kQBytes + kPBytes;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -271,7 +271,8 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     // ---- set-up
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(&hd->kv_full[i], 1); mbar_init(&hd->kv_empty[i], 1); }
-        mbar_init(&hd->q_full, 1); mbar_init(&hd->q_empty, 1);
+        mbar_init(&hd->q_full[0], 1); mbar_init(&hd->q_full[1], 1);
+        mbar_init(&hd->q_empty[0], 1); mbar_init(&hd->q_empty[1], 1);
         mbar_init(&hd->s_full[0], 1); mbar_init(&hd->s_full[1], 1);
         mbar_init(&hd->p_ready, 128); mbar_init(&hd->pv_done, 1); mbar_init(&hd->o_free, 128);
         mbar_init(&hd->group_bar, 128);
@@ -287,6 +288,9 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = hd->tmem_base;
+    // let the combine kernel (launched with programmatic stream serialisation) get resident early; it
+    // still waits for this grid to finish before it reads the partials
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (w_begin < w_end) {
         if (warp == 0) {
@@ -304,11 +308,12 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 while (ok && cu.w < w_end) {
                     const int64_t row0 = row_off[cu.s];
                     // Q of this segment
-                    ok = mbar_wait(hd, &hd->q_empty, (seg & 1) ^ 1, status);   // seg = index of this segment
+                    const uint32_t qb = seg & 1;           // seg = index of this segment
+                    ok = mbar_wait(hd, &hd->q_empty[qb], ((seg >> 1) & 1) ^ 1, status);
                     if (!ok) break;
-                    mbar_expect_tx(&hd->q_full, (uint32_t)B * 256u);
-                    tma_load_3d(q_smem, &tmap_q, &hd->q_full, 0, cu.h, cu.s * B);
-                    tma_load_3d(q_smem + kHalfBytes, &tmap_q, &hd->q_full, 64, cu.h, cu.s * B);
+                    mbar_expect_tx(&hd->q_full[qb], (uint32_t)B * 256u);
+                    tma_load_3d(q_smem + qb * kQBytes, &tmap_q, &hd->q_full[qb], 0, cu.h, cu.s * B);
+                    tma_load_3d(q_smem + qb * kQBytes + kHalfBytes, &tmap_q, &hd->q_full[qb], 64, cu.h, cu.s * B);
                     ++seg;                                 // segments whose Q load has been issued
                     const int s0 = cu.s, h0 = cu.h;
                     while (ok && cu.w < w_end && cu.s == s0 && cu.h == h0) {
@@ -332,7 +337,8 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                     // aborted: drain this thread's copies still in flight (bounded) before the CTA exits
                     uint32_t first = ring > kStages ? ring - kStages : 0;
                     for (uint32_t r = first; r < ring; ++r) mbar_drain(&hd->kv_full[r % kStages], (r / kStages) & 1);
-                    if (seg > 0) mbar_drain(&hd->q_full, (seg - 1) & 1);
+                    if (seg > 0) mbar_drain(&hd->q_full[(seg - 1) & 1], ((seg - 1) >> 1) & 1);
+                    if (seg > 1) mbar_drain(&hd->q_full[(seg - 2) & 1], ((seg - 2) >> 1) & 1);
                 }
             }
         } else if (warp == 1) {
@@ -343,7 +349,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 bool ok = true;
                 int tn = 0; (void)tn;
                 TRACE(1, tn, 1);
-                const uint32_t q_addr = smem_u32(q_smem), p_addr = smem_u32(p_smem), kv_addr = smem_u32(kv_smem);
+                const uint32_t q_base = smem_u32(q_smem), p_addr = smem_u32(p_smem), kv_addr = smem_u32(kv_smem);
                 constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
 
                 auto issue_pv = [&](uint32_t j, bool first_of_segment) -> bool {
@@ -368,8 +374,9 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 };
 
                 while (ok && cu.w < w_end) {
-                    ok = mbar_wait(hd, &hd->q_full, seg & 1, status);
+                    ok = mbar_wait(hd, &hd->q_full[seg & 1], (seg >> 1) & 1, status);
                     if (!ok) break;
+                    const uint32_t q_addr = q_base + (seg & 1) * kQBytes;
                     const int s0 = cu.s, h0 = cu.h;
                     const uint32_t j_first = jg;
                     while (ok && cu.w < w_end && cu.s == s0 && cu.h == h0) {
@@ -393,7 +400,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                         cu.next(wk);
                     }
                     if (!ok) break;
-                    umma_commit(&hd->q_empty);             // every QK^T of the segment has been issued
+                    umma_commit(&hd->q_empty[seg & 1]);    // every QK^T of the segment has been issued
                     ok = issue_pv(jg - 1, jg - 1 == j_first);
                     ++seg;
                 }
@@ -408,6 +415,9 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
             uint32_t jg = 0, seg = 0, gsync = 0;
             bool ok = true;
             uint32_t v[128];
+            int cur_s = -1;
+            bool bad = false;
+            uint32_t anc[4] = {0, 0, 0, 0};
             int tn = 0; (void)tn;
             if (sm_tid == 0) TRACE(2, tn, 1);
 
@@ -417,29 +427,33 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 const int n_keys = ctx + B;
                 const int32_t* par = parent + (size_t)s0 * B;
                 const int t_first = cu.t;
-                // validate parent[] of this sequence (all 128 threads reach the same verdict)
-                if (row < B) {
-                    int p = par[row];
-                    hd->par[row] = p;
-                    if ((row == 0) ? (p != -1) : (p < 0 || p >= row)) hd->bad_parent = 1;
-                }
-                ok = group_sync(hd, gsync, status);
-                const bool bad = hd->bad_parent != 0;
-                ok = ok && group_sync(hd, gsync, status);
-                if (!ok) break;
-                if (sm_tid == 0 && bad) { hd->bad_parent = 0; atomicOr(&status[s0], GOOSE_ST_BAD_PARENT); }
-                uint32_t anc[4] = {0, 0, 0, 0};
-                if (row < B) {
-                    if (bad) {
-                        anc[row >> 5] = 1u << (row & 31);
-                    } else {
-                        int vtx = row;
-                        for (int step = 0; step < B && vtx >= 0; ++step) {
-                            uint32_t bit = 1u << (vtx & 31);
-                            int wsel = vtx >> 5;
-                            anc[0] |= (wsel == 0) ? bit : 0; anc[1] |= (wsel == 1) ? bit : 0;
-                            anc[2] |= (wsel == 2) ? bit : 0; anc[3] |= (wsel == 3) ? bit : 0;
-                            vtx = hd->par[vtx];
+                // new sequence: validate parent[] (all 128 threads reach the same verdict) and rebuild
+                // this row's ancestor set; consecutive segments of one sequence reuse both
+                if (s0 != cur_s) {
+                    cur_s = s0;
+                    if (row < B) {
+                        int p = par[row];
+                        hd->par[row] = p;
+                        if ((row == 0) ? (p != -1) : (p < 0 || p >= row)) hd->bad_parent = 1;
+                    }
+                    ok = group_sync(hd, gsync, status);
+                    bad = hd->bad_parent != 0;
+                    ok = ok && group_sync(hd, gsync, status);
+                    if (!ok) break;
+                    if (sm_tid == 0 && bad) { hd->bad_parent = 0; atomicOr(&status[s0], GOOSE_ST_BAD_PARENT); }
+                    anc[0] = anc[1] = anc[2] = anc[3] = 0;
+                    if (row < B) {
+                        if (bad) {
+                            anc[row >> 5] = 1u << (row & 31);
+                        } else {
+                            int vtx = row;
+                            for (int step = 0; step < B && vtx >= 0; ++step) {
+                                uint32_t bit = 1u << (vtx & 31);
+                                int wsel = vtx >> 5;
+                                anc[0] |= (wsel == 0) ? bit : 0; anc[1] |= (wsel == 1) ? bit : 0;
+                                anc[2] |= (wsel == 2) ? bit : 0; anc[3] |= (wsel == 3) ? bit : 0;
+                                vtx = hd->par[vtx];
+                            }
                         }
                     }
                 }
@@ -645,6 +659,7 @@ tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, const int32_t* __r
     const long long head_first = off + (long long)h * T;
     const int c_lo = wk.cta_of(head_first), c_hi = wk.cta_of(head_first + T - 1);
     if (c_lo == c_hi) return;                              // written directly by the main kernel
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // the main kernel's partials are complete and visible
     // invalid parent[] -> zero-filled output (the main kernel has already set the status word)
     int bad = 0;
     for (int i = tid; i < B; i += 128) {
@@ -784,9 +799,16 @@ cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     dim3 cgrid((B + 31) / 32, H, S);
-    tree_attn_combine_kernel<<<cgrid, 128, 0, st>>>(ctx_len, parent, S, B, H, grid, c->partials, out, lse);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = cgrid; cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    const float* parts = c->partials;
+    e = cudaLaunchKernelEx(&cfg, tree_attn_combine_kernel, ctx_len, parent, S, B, H, grid, parts, out, lse);
     c->launches++;
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace goose

@@ -18,6 +18,8 @@ accept_kernel(const int32_t* __restrict__ draft_tok, const int32_t* __restrict__
     const int32_t* tok = draft_tok + (size_t)s * B;
     const int32_t* am = argmax + (size_t)s * B;
     int32_t* p = path + (size_t)s * B;
+    pdl_wait();
+    pdl_trigger();
 
     constexpr int kPer = kMaxB / 32;
     int my_par[kPer];
@@ -72,9 +74,10 @@ accept_kernel(const int32_t* __restrict__ draft_tok, const int32_t* __restrict__
 cudaError_t launch_accept(goose_ctx* c, const int32_t* draft_tok, const int32_t* parent, const int32_t* argmax,
                           int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus, cudaStream_t st) {
     if (S == 0) return cudaSuccess;
-    accept_kernel<<<S, 32, 0, st>>>(draft_tok, parent, argmax, B, path, accept_len, bonus, c->status);
+    cudaError_t e = launch_pdl(accept_kernel, dim3(S), dim3(32), 0, st, draft_tok, parent, argmax, B, path,
+                               accept_len, bonus, c->status);
     c->launches++;
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace goose

@@ -43,6 +43,29 @@ struct goose_ctx {
 
 namespace goose {
 
+// Programmatic dependent launch.  Every kernel of the library is launched with the
+// programmatic-stream-serialisation attribute and runs  prologue (no global memory access) ->
+// pdl_wait() -> pdl_trigger() -> body.  pdl_wait() returns once the preceding kernel in the stream has
+// completed and its writes are visible; because that kernel passed its own pdl_wait() before it
+// triggered, completion is transitive over the whole stream.  The overlap gained is the launch latency
+// and the prologue of the next kernel.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
+
 // launchers (each returns a cudaError_t from the launch)
 cudaError_t launch_node_topk(goose_ctx* c, const __nv_bfloat16* logits, int rows, int V, int64_t ldl, int k,
                              int32_t* argmax, int32_t* ids, float* vals, cudaStream_t st);

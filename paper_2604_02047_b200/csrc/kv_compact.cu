@@ -14,7 +14,7 @@ constexpr int kCompactThreads = 128;
 constexpr int kCompactBatch = 8;
 
 __global__ void __launch_bounds__(kCompactThreads)
-kv_compact_kernel(__nv_bfloat16* __restrict__ kc, __nv_bfloat16* __restrict__ vc,
+kv_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc,
                   const int64_t* __restrict__ row_off, const int32_t* __restrict__ ctx_len,
                   const int32_t* __restrict__ path, const int32_t* __restrict__ accept_len,
                   int B, int row_vec /* 16-byte vectors per row = H*128*2/16 */,
@@ -24,6 +24,8 @@ kv_compact_kernel(__nv_bfloat16* __restrict__ kc, __nv_bfloat16* __restrict__ vc
     const int s = blockIdx.z;
     const int which = blockIdx.y;                        // 0 = K, 1 = V
     const int col = blockIdx.x * kCompactThreads + threadIdx.x;
+    pdl_wait();
+    pdl_trigger();
     const int ctx = ctx_len[s];
     int L = accept_len[s];
     if (threadIdx.x == 0) s_bad = 0;
@@ -68,10 +70,10 @@ cudaError_t launch_kv_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc
     if (S == 0) return cudaSuccess;
     int row_vec = H * kHeadDim * 2 / 16;
     dim3 grid((row_vec + kCompactThreads - 1) / kCompactThreads, 2, S);
-    kv_compact_kernel<<<grid, kCompactThreads, 0, st>>>(kc, vc, row_off, ctx_len, path, accept_len, B, row_vec,
-                                                        new_ctx, c->status);
+    cudaError_t e = launch_pdl(kv_compact_kernel, grid, dim3(kCompactThreads), 0, st, kc, vc, row_off, ctx_len, path,
+                               accept_len, B, row_vec, new_ctx, c->status);
     c->launches++;
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace goose

@@ -1,13 +1,16 @@
 // Per-node argmax and top-k over bf16 logits (Algorithm 3 step 2; batched top-K harvest of App. C.1).
 //
 // A row is cut into chunks of 32768 elements; one 1024-thread CTA scans one chunk with 128-bit loads
-// held in registers (32 values per thread).  Inside a chunk every element is a 32-bit key
+// held in registers (32 values per thread).  The exact order is carried by 32-bit keys
 //     (order-preserving 16-bit image of the bf16 value) << 16 | (0xFFFF - index_in_chunk)
 // so "largest key" is "largest value, lowest index on ties", all keys are distinct, and a key carries
-// its own index.  Warp-wide maxima are single redux.sync instructions: each warp extracts its k best
-// in k rounds (only the lane that owned the winner rescans its registers), warp 0 then selects the
-// chunk's k best from the 32*k candidates.  Rows longer than one chunk (V > 32768) finish with a merge
-// of the chunks' candidates by the last CTA to arrive for the row (arrival counter, no spinning).
+// its own index.  Building a key costs several instructions per element, so keys are built only for
+// candidates: packed-bf16 maxima give every thread's maximum, redux.sync rounds give the k-th largest
+// thread maximum T of the CTA (every top-k element is >= T), and only the elements >= T (about k of
+// 32768) are turned into keys and ranked by one warp.  Rows with more than 1024 elements tied at or
+// above T (a constant row) take an exact slow path over all keys.  Rows longer than one chunk
+// (V > 32768) finish with a merge of the chunks' candidates by the last CTA to arrive for the row
+// (arrival counter, no spinning).
 #include "goose_internal.cuh"
 
 namespace goose {
@@ -30,11 +33,16 @@ __device__ __forceinline__ float value_of_sortable16(uint32_t s) {
     return __uint_as_float(bits << 16);
 }
 
-__device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
+// 8 consecutive bf16 of a row starting at element idx (a multiple of 8); elements past V read as -inf.
+// Plain cached loads: the row chunk is read a second time (from L1/L2) once the threshold is known,
+// which keeps the 32 values per thread out of the register file between the two passes.
+__device__ __forceinline__ uint4 load8(const unsigned short* rowp, int idx, int V) {
+    if (idx + 8 <= V) return __ldg(reinterpret_cast<const uint4*>(rowp + idx));
+    unsigned short t[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) t[e] = (idx + e < V) ? rowp[idx + e] : (unsigned short)0xFF80u;
+    return make_uint4(t[0] | ((uint32_t)t[1] << 16), t[2] | ((uint32_t)t[3] << 16),
+                      t[4] | ((uint32_t)t[5] << 16), t[6] | ((uint32_t)t[7] << 16));
 }
 
 __device__ __forceinline__ u64 warp_max_u64(u64 v) {
@@ -46,13 +54,24 @@ __device__ __forceinline__ u64 warp_max_u64(u64 v) {
     return v;
 }
 
+constexpr int kTopkListCap = 1024;                           // candidate list of the fast path
+
+__device__ __forceinline__ uint32_t bits_of_sortable16(uint32_t s) {
+    return (s & 0x8000u) ? (s ^ 0x8000u) : (~s & 0xFFFFu);
+}
+__device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t w) { return *reinterpret_cast<__nv_bfloat162*>(&w); }
+__device__ __forceinline__ uint32_t as_u32(__nv_bfloat162 v) { return *reinterpret_cast<uint32_t*>(&v); }
+
 template <int KCAP>
-__global__ void __launch_bounds__(kTopkThreads, 1)
+__global__ void __launch_bounds__(kTopkThreads, 2)
 node_topk_kernel(const __nv_bfloat16* __restrict__ logits, int V, int64_t ldl, int k, int chunks,
                  u64* __restrict__ ws_cand, int32_t* __restrict__ row_counters,
                  int32_t* __restrict__ argmax, int32_t* __restrict__ ids, float* __restrict__ vals) {
-    __shared__ uint32_t s_cand[32 * KCAP];
+    __shared__ uint32_t s_cand[32 * KCAP];               // per-warp winners (thread maxima, or exact keys)
+    __shared__ uint32_t s_list[kTopkListCap];            // fast path: keys of all elements >= threshold
     __shared__ u64 s_merge[kTopkMaxChunks * KCAP];
+    __shared__ uint32_t s_thresh;
+    __shared__ int s_count;
     __shared__ int s_last;
 
     const int row = blockIdx.y;
@@ -60,74 +79,148 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, int V, int64_t ldl, i
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned short* rowp = reinterpret_cast<const unsigned short*>(logits) + (size_t)row * ldl;
     const int base = chunk * kTopkChunk;
+    if (tid == 0) s_count = 0;
+    pdl_wait();
+    pdl_trigger();
 
-    // ---- 32 values per thread: element (it, e) of thread tid sits at chunk offset it*8192 + tid*8 + e
-    uint4 raw[4];
+    // ---- phase 1: 32 values per thread (element (it, e) of thread tid sits at chunk offset
+    //      it*8192 + tid*8 + e); thread maximum with packed bf16 max
+    __nv_bfloat162 m2;
+    {
+        uint4 v4[4];
 #pragma unroll
-    for (int it = 0; it < 4; ++it) {
-        int idx = base + it * (kTopkThreads * 8) + tid * 8;
-        if (idx + 8 <= V) {
-            raw[it] = ldg_stream(reinterpret_cast<const uint4*>(rowp + idx));
-        } else {
-            unsigned short t[8];
+        for (int it = 0; it < 4; ++it) v4[it] = load8(rowp, base + it * (kTopkThreads * 8) + tid * 8, V);
+        m2 = __hmax2(as_bf162(v4[0].x), as_bf162(v4[0].y));
+        m2 = __hmax2(m2, __hmax2(as_bf162(v4[0].z), as_bf162(v4[0].w)));
 #pragma unroll
-            for (int e = 0; e < 8; ++e) t[e] = (idx + e < V) ? rowp[idx + e] : (unsigned short)0;
-            raw[it].x = t[0] | ((uint32_t)t[1] << 16); raw[it].y = t[2] | ((uint32_t)t[3] << 16);
-            raw[it].z = t[4] | ((uint32_t)t[5] << 16); raw[it].w = t[6] | ((uint32_t)t[7] << 16);
+        for (int it = 1; it < 4; ++it) {
+            m2 = __hmax2(m2, __hmax2(as_bf162(v4[it].x), as_bf162(v4[it].y)));
+            m2 = __hmax2(m2, __hmax2(as_bf162(v4[it].z), as_bf162(v4[it].w)));
         }
     }
-    uint32_t key[kTopkPerThread];
-    uint32_t best = 0;
-#pragma unroll
-    for (int it = 0; it < 4; ++it) {
-        int off = it * (kTopkThreads * 8) + tid * 8;
-        uint32_t w[4] = {raw[it].x, raw[it].y, raw[it].z, raw[it].w};
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            uint32_t bits = (e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu);
-            uint32_t kk = (base + off + e < V) ? ((sortable16(bits) << 16) | (0xFFFFu - (uint32_t)(off + e))) : 0u;
-            key[it * 8 + e] = kk;
-            best = kk > best ? kk : best;
-        }
-    }
+    const uint32_t mw = as_u32(m2);
+    const uint32_t s_lo = sortable16(mw & 0xFFFFu), s_hi = sortable16(mw >> 16);
+    uint32_t tmax = s_lo > s_hi ? s_lo : s_hi;
 
-    // ---- each warp extracts its k best (redux.sync max; the owning lane drops the winner and rescans)
+    // ---- phase 2: each warp lists its k largest thread maxima (descending; equal maxima are kept)
     for (int r = 0; r < k; ++r) {
-        uint32_t w = __reduce_max_sync(0xFFFFFFFFu, best);
+        const uint32_t w = __reduce_max_sync(0xFFFFFFFFu, tmax);
+        const uint32_t owners = __ballot_sync(0xFFFFFFFFu, tmax == w);
         if (lane == 0) s_cand[warp * KCAP + r] = w;
-        if (best == w && w != 0) {
-            uint32_t nb = 0;
-#pragma unroll
-            for (int j = 0; j < kTopkPerThread; ++j) {
-                key[j] = (key[j] == w) ? 0u : key[j];
-                nb = key[j] > nb ? key[j] : nb;
+        if (lane == __ffs(owners) - 1) tmax = 0;
+    }
+    __syncthreads();
+
+    // ---- phase 3: warp 0 finds T = the k-th largest thread maximum of the CTA.  At least k elements are
+    //      >= T, hence every one of the chunk's k best is >= T.
+    if (warp == 0) {
+        int ptr = 0;                                     // lane l walks warp l's sorted list
+        uint32_t cur = s_cand[lane * KCAP];
+        uint32_t w = 0;
+        for (int r = 0; r < k; ++r) {
+            w = __reduce_max_sync(0xFFFFFFFFu, cur);
+            const uint32_t owners = __ballot_sync(0xFFFFFFFFu, cur == w);
+            if (lane == __ffs(owners) - 1) {
+                ++ptr;
+                cur = ptr < k ? s_cand[lane * KCAP + ptr] : 0u;
             }
-            best = nb;
+        }
+        if (lane == 0) s_thresh = w;
+    }
+    __syncthreads();
+
+    // ---- phase 4: every element >= T becomes a full key (value image << 16 | 0xFFFF - index in chunk)
+    const uint32_t thr_s = s_thresh;
+    {
+        const uint32_t tb = bits_of_sortable16(thr_s);
+        const __nv_bfloat162 t2 = as_bf162(tb | (tb << 16));
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const uint4 v4 = load8(rowp, base + it * (kTopkThreads * 8) + tid * 8, V);
+            const uint32_t wds[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t ge = __hge2_mask(as_bf162(wds[q]), t2);
+                if (ge) {
+                    const int off = it * (kTopkThreads * 8) + tid * 8 + q * 2;
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        if (((ge >> (16 * e)) & 1u) && base + off + e < V) {
+                            const uint32_t bits = e ? (wds[q] >> 16) : (wds[q] & 0xFFFFu);
+                            const int pos = atomicAdd(&s_count, 1);
+                            if (pos < kTopkListCap) s_list[pos] = (sortable16(bits) << 16) | (0xFFFFu - (uint32_t)(off + e));
+                        }
+                    }
+                }
+            }
         }
     }
     __syncthreads();
-    if (warp != 0) return;
+    const int n_list = s_count;
 
-    // ---- warp 0: the chunk's k best out of 32 warps x k candidates (one warp's list per lane)
-    uint32_t c[KCAP];
-    uint32_t lm = 0;
-#pragma unroll
-    for (int j = 0; j < KCAP; ++j) {
-        c[j] = (j < k) ? s_cand[lane * KCAP + j] : 0u;       // sorted descending within a lane
-        lm = c[j] > lm ? c[j] : lm;
-    }
-    uint32_t mine = 0;                                       // lane r keeps the r-th winner
-    for (int r = 0; r < k; ++r) {
-        uint32_t w = __reduce_max_sync(0xFFFFFFFFu, lm);
-        if (lane == r) mine = w;
-        if (lm == w && w != 0) {
+    uint32_t mine = 0;                                   // warp 0: lane r ends up with the r-th winner
+    if (n_list <= kTopkListCap) {
+        // ---- phase 5 (fast path): warp 0 selects the k best of the list
+        if (warp != 0) return;
+        for (int r = 0; r < k; ++r) {
+            uint32_t m = 0;
+            for (int j = lane; j < n_list; j += 32) m = s_list[j] > m ? s_list[j] : m;
+            const uint32_t w = __reduce_max_sync(0xFFFFFFFFu, m);
+            if (lane == r) mine = w;
+            if (w != 0)
+                for (int j = lane; j < n_list; j += 32)
+                    if (s_list[j] == w) s_list[j] = 0;
+            __syncwarp();
+        }
+    } else {
+        // ---- slow path (more than kTopkListCap elements tie at or above T, e.g. a constant row):
+        //      exact rounds on full keys of all 32 values per thread
+        //      exact rounds on full keys, rebuilt from the (cached) row whenever a lane needs its next best
+        // largest key of this thread strictly below `bound` (all keys are distinct)
+        auto best_below = [&](uint32_t bound) -> uint32_t {
             uint32_t nb = 0;
 #pragma unroll
-            for (int j = 0; j < KCAP; ++j) {
-                c[j] = (c[j] == w) ? 0u : c[j];
-                nb = c[j] > nb ? c[j] : nb;
+            for (int it = 0; it < 4; ++it) {
+                const int off0 = it * (kTopkThreads * 8) + tid * 8;
+                const uint4 v4 = load8(rowp, base + off0, V);
+                const uint32_t wds[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const uint32_t bits = (e & 1) ? (wds[e >> 1] >> 16) : (wds[e >> 1] & 0xFFFFu);
+                    const uint32_t kk = (base + off0 + e < V) ? ((sortable16(bits) << 16) | (0xFFFFu - (uint32_t)(off0 + e))) : 0u;
+                    nb = (kk < bound && kk > nb) ? kk : nb;
+                }
             }
-            lm = nb;
+            return nb;
+        };
+        uint32_t best = best_below(0xFFFFFFFFu);
+        __syncthreads();                                 // s_cand is reused
+        for (int r = 0; r < k; ++r) {
+            const uint32_t w = __reduce_max_sync(0xFFFFFFFFu, best);
+            if (lane == 0) s_cand[warp * KCAP + r] = w;
+            if (best == w && w != 0) best = best_below(w);
+        }
+        __syncthreads();
+        if (warp != 0) return;
+        uint32_t c[KCAP];
+        uint32_t lm = 0;
+#pragma unroll
+        for (int j = 0; j < KCAP; ++j) {
+            c[j] = (j < k) ? s_cand[lane * KCAP + j] : 0u;
+            lm = c[j] > lm ? c[j] : lm;
+        }
+        for (int r = 0; r < k; ++r) {
+            uint32_t w = __reduce_max_sync(0xFFFFFFFFu, lm);
+            if (lane == r) mine = w;
+            if (lm == w && w != 0) {
+                uint32_t nb = 0;
+#pragma unroll
+                for (int j = 0; j < KCAP; ++j) {
+                    c[j] = (c[j] == w) ? 0u : c[j];
+                    nb = c[j] > nb ? c[j] : nb;
+                }
+                lm = nb;
+            }
         }
     }
     int32_t my_id = base + (int32_t)(0xFFFFu - (mine & 0xFFFFu));
@@ -182,14 +275,9 @@ cudaError_t launch_node_topk(goose_ctx* c, const __nv_bfloat16* logits, int rows
         const __nv_bfloat16* lp = logits + (size_t)r0 * ldl;
         u64* ws = c->topk_cand + (size_t)r0 * chunks * kMaxK;
         float* vp = vals ? vals + (size_t)r0 * k : nullptr;
-        if (k <= 8)
-            node_topk_kernel<8><<<grid, kTopkThreads, 0, st>>>(lp, V, ldl, k, chunks, ws, c->row_counters + r0,
-                                                              argmax + r0, ids + (size_t)r0 * k, vp);
-        else
-            node_topk_kernel<16><<<grid, kTopkThreads, 0, st>>>(lp, V, ldl, k, chunks, ws, c->row_counters + r0,
-                                                               argmax + r0, ids + (size_t)r0 * k, vp);
+        cudaError_t e = launch_pdl(k <= 8 ? node_topk_kernel<8> : node_topk_kernel<16>, grid, dim3(kTopkThreads), 0, st,
+                                   lp, V, ldl, k, chunks, ws, c->row_counters + r0, argmax + r0, ids + (size_t)r0 * k, vp);
         c->launches++;
-        cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;

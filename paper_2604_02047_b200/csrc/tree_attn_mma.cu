@@ -96,6 +96,8 @@ tree_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     const int split = blockIdx.x, h = blockIdx.y, s = blockIdx.z;
     const int tid = threadIdx.x, nthreads = blockDim.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, t4 = lane & 3;
+    pdl_wait();
+    pdl_trigger();
     const int ctx = ctx_len[s];
     const int64_t row0 = row_off[s];
     const int n_keys = ctx + B;
@@ -322,11 +324,10 @@ cudaError_t launch_tree_attn_mma(goose_ctx* c, const __nv_bfloat16* q, const __n
     int warps = (B + 15) / 16;
     if (warps < 4) warps = 4;
     dim3 grid(splits, H, S);
-    tree_attn_mma_kernel<<<grid, warps * 32, kMmaSmem, st>>>(q, kc, vc, row_off, ctx_len, parent, B, H,
-                                                           scale * kLog2e, splits, c->partials, c->head_counters,
-                                                           c->status, out, lse);
+    cudaError_t e = launch_pdl(tree_attn_mma_kernel, grid, dim3(warps * 32), kMmaSmem, st, q, kc, vc, row_off, ctx_len,
+                               parent, B, H, scale * kLog2e, splits, c->partials, c->head_counters, c->status, out, lse);
     c->launches++;
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace goose

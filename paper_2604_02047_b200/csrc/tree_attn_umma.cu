@@ -44,6 +44,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;       // rescale O only when the running max grew by > 2^8
 constexpr int kCombineChunk = 8;                 // partials merged per pass of the combine kernel
+constexpr int kCombineThreads = 256;
 constexpr long long kWaitCycles = 2000000000ll;  // bound of every wait: about one second of SM clock
 
 #ifdef GOOSE_TRACE
@@ -58,8 +59,10 @@ __device__ __forceinline__ void trace_ev(int role, int& n, unsigned tag) {
     }
 }
 #define TRACE(role, n, tag) trace_ev(role, n, tag)
+#define TRACE_DECL int tn = 0
 #else
 #define TRACE(role, n, tag) do { } while (0)
+#define TRACE_DECL do { } while (0)
 #endif
 
 struct Header {                                  // lives at the start of dynamic shared memory
@@ -259,15 +262,6 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    Work wk;
-    wk.ctx_len = ctx_len; wk.S = S; wk.H = H; wk.B = B; wk.G = gridDim.x;
-    {
-        long long tot = 0;
-        for (int s = 0; s < S; ++s) tot += (long long)H * wk.tiles(s);
-        wk.total = tot;
-    }
-    const long long w_begin = wk.cta_start(blockIdx.x), w_end = wk.cta_start(blockIdx.x + 1);
-
     // ---- set-up
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(&hd->kv_full[i], 1); mbar_init(&hd->kv_empty[i], 1); }
@@ -288,9 +282,19 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = hd->tmem_base;
-    // let the combine kernel (launched with programmatic stream serialisation) get resident early; it
-    // still waits for this grid to finish before it reads the partials
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // everything above touched no global memory: now wait for the preceding kernel, then let the next
+    // one (the combine kernel) get resident early -- it waits for this grid before reading the partials
+    pdl_wait();
+    pdl_trigger();
+    Work wk;
+    wk.ctx_len = ctx_len; wk.S = S; wk.H = H; wk.B = B; wk.G = gridDim.x;
+    {
+        long long tot = 0;
+        for (int s = 0; s < S; ++s) tot += (long long)H * wk.tiles(s);
+        wk.total = tot;
+    }
+    const long long w_begin = wk.cta_start(blockIdx.x), w_end = wk.cta_start(blockIdx.x + 1);
+
 
     if (w_begin < w_end) {
         if (warp == 0) {
@@ -303,7 +307,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 Cursor cu; cu.seek(wk, w_begin);
                 uint32_t ring = 0, seg = 0;
                 bool ok = true;
-                int tn = 0; (void)tn;
+                TRACE_DECL;
                 TRACE(0, tn, 1);
                 while (ok && cu.w < w_end) {
                     const int64_t row0 = row_off[cu.s];
@@ -347,7 +351,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 Cursor cu; cu.seek(wk, w_begin);
                 uint32_t jg = 0, seg = 0;                  // CTA-global tile and segment counters
                 bool ok = true;
-                int tn = 0; (void)tn;
+                TRACE_DECL;
                 TRACE(1, tn, 1);
                 const uint32_t q_base = smem_u32(q_smem), p_addr = smem_u32(p_smem), kv_addr = smem_u32(kv_smem);
                 constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
@@ -418,7 +422,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
             int cur_s = -1;
             bool bad = false;
             uint32_t anc[4] = {0, 0, 0, 0};
-            int tn = 0; (void)tn;
+            TRACE_DECL;
             if (sm_tid == 0) TRACE(2, tn, 1);
 
             while (ok && cu.w < w_end) {
@@ -636,17 +640,19 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
 }
 
 // ---------------------------------------------------------------- combine of the split-KV partials
-// Grid (row groups of 32, H, S), 128 threads.  A head that one CTA of the main kernel covered entirely
+// Grid (row groups of 32, H, S), 256 threads.  A head that one CTA of the main kernel covered entirely
 // was written directly and is skipped; any other head is the merge of its CTAs' partials:
 //   M = max m_p,  L = sum l_p 2^(m_p - M),  out = sum_p 2^(m_p - M) O_p / L.
-// Lane <-> row (coalesced float4 loads of the transposed partial layout), warp <-> 32 output columns.
-__global__ void __launch_bounds__(128)
+// Lane <-> row (coalesced float4 loads of the transposed partial layout), warp <-> 16 output columns.
+__global__ void __launch_bounds__(kCombineThreads)
 tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ parent,
                          int S, int B, int H, int G, const float* __restrict__ partials,
                          __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
     __shared__ int slot_s[kCombineChunk];
     const int rg = blockIdx.x, h = blockIdx.y, s = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pdl_wait();                                            // the main kernel's partials are complete and visible
+    pdl_trigger();
     Work wk;
     wk.ctx_len = ctx_len; wk.S = S; wk.H = H; wk.B = B; wk.G = G;
     long long tot = 0, off = 0;
@@ -659,20 +665,20 @@ tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, const int32_t* __r
     const long long head_first = off + (long long)h * T;
     const int c_lo = wk.cta_of(head_first), c_hi = wk.cta_of(head_first + T - 1);
     if (c_lo == c_hi) return;                              // written directly by the main kernel
-    asm volatile("griddepcontrol.wait;" ::: "memory");     // the main kernel's partials are complete and visible
     // invalid parent[] -> zero-filled output (the main kernel has already set the status word)
     int bad = 0;
-    for (int i = tid; i < B; i += 128) {
+    for (int i = tid; i < B; i += kCombineThreads) {
         int p = parent[(size_t)s * B + i];
         bad |= (i == 0) ? (p != -1) : (p < 0 || p >= i);
     }
     bad = __syncthreads_or(bad);
     const int row = rg * 32 + lane;
     const bool row_ok = row < B;
+    const int rr = row_ok ? row : 0;
     float M_run = -INFINITY, L_run = 0.f;
-    float4 acc[8];
+    float4 acc[4];                                         // warp w owns column groups 4w .. 4w+3 (16 columns)
 #pragma unroll
-    for (int u = 0; u < 8; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
 
     // parts in chunks; a running (M, L) with rescaling of the accumulators keeps chunks independent
     for (int cb = c_lo; cb <= c_hi; cb += kCombineChunk) {
@@ -687,7 +693,6 @@ tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, const int32_t* __r
             slot_s[tid] = sl;
         }
         __syncthreads();
-        // this chunk's row statistics (every warp computes them for its own lanes' rows)
         float mp[kCombineChunk], lp[kCombineChunk];
 #pragma unroll
         for (int pi = 0; pi < kCombineChunk; ++pi) {
@@ -703,40 +708,41 @@ tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, const int32_t* __r
         const float a_old = (M_run == -INFINITY) ? 0.f : ex2(M_run - M_new);
         L_run *= a_old;
 #pragma unroll
-        for (int u = 0; u < 8; ++u) { acc[u].x *= a_old; acc[u].y *= a_old; acc[u].z *= a_old; acc[u].w *= a_old; }
+        for (int u = 0; u < 4; ++u) { acc[u].x *= a_old; acc[u].y *= a_old; acc[u].z *= a_old; acc[u].w *= a_old; }
 #pragma unroll
         for (int pi = 0; pi < kCombineChunk; ++pi) {
             const float w = (mp[pi] == -INFINITY) ? 0.f : ex2(mp[pi] - M_new);
             L_run += w * lp[pi];
-            mp[pi] = w;                                    // reuse as the part's weight for this row
+            mp[pi] = w;                                    // from here on: the part's weight for this row
         }
         M_run = M_new;
-        // accumulate: warp w owns column groups 8w .. 8w+7 (32 output columns)
 #pragma unroll
-        for (int pi = 0; pi < kCombineChunk; pi += 2) {
-            const int sl0 = slot_s[pi], sl1 = slot_s[pi + 1];
-            if (sl0 < 0 && sl1 < 0) continue;             // uniform over the CTA
-            const float4* p0 = reinterpret_cast<const float4*>(partials + (size_t)(sl0 < 0 ? 0 : sl0) * kPartialFloats) + (row_ok ? row : 0);
-            const float4* p1 = reinterpret_cast<const float4*>(partials + (size_t)(sl1 < 0 ? 0 : sl1) * kPartialFloats) + (row_ok ? row : 0);
-            float4 x0[8], x1[8];
+        for (int p0 = 0; p0 < kCombineChunk; p0 += 4) {    // four parts = 16 independent 16-byte loads in flight
+            if (slot_s[p0] < 0 && slot_s[p0 + 1] < 0 && slot_s[p0 + 2] < 0 && slot_s[p0 + 3] < 0) continue;
+            float4 x[4][4];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                x0[u] = __ldcg(p0 + (8 * warp + u) * 128);
-                x1[u] = __ldcg(p1 + (8 * warp + u) * 128);
+            for (int q = 0; q < 4; ++q) {
+                const int sl = slot_s[p0 + q];
+                const float4* pp = reinterpret_cast<const float4*>(partials + (size_t)(sl < 0 ? 0 : sl) * kPartialFloats) + rr;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) x[q][u] = __ldcg(pp + (4 * warp + u) * 128);
             }
-            const float w0 = sl0 < 0 ? 0.f : mp[pi], w1 = sl1 < 0 ? 0.f : mp[pi + 1];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                acc[u].x += w0 * x0[u].x + w1 * x1[u].x; acc[u].y += w0 * x0[u].y + w1 * x1[u].y;
-                acc[u].z += w0 * x0[u].z + w1 * x1[u].z; acc[u].w += w0 * x0[u].w + w1 * x1[u].w;
+            for (int q = 0; q < 4; ++q) {
+                const float w = slot_s[p0 + q] < 0 ? 0.f : mp[p0 + q];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    acc[u].x += w * x[q][u].x; acc[u].y += w * x[q][u].y;
+                    acc[u].z += w * x[q][u].z; acc[u].w += w * x[q][u].w;
+                }
             }
         }
     }
     if (!row_ok) return;
     const float inv = bad ? 0.f : 1.f / L_run;
-    uint4* dst = reinterpret_cast<uint4*>(out + (((size_t)s * B + row) * H + h) * kHeadDim + 32 * warp);
+    uint4* dst = reinterpret_cast<uint4*>(out + (((size_t)s * B + row) * H + h) * kHeadDim + 16 * warp);
 #pragma unroll
-    for (int u = 0; u < 8; u += 2)
+    for (int u = 0; u < 4; u += 2)
         dst[u >> 1] = make_uint4(pack_bf16x2(acc[u].x * inv, acc[u].y * inv), pack_bf16x2(acc[u].z * inv, acc[u].w * inv),
                                  pack_bf16x2(acc[u + 1].x * inv, acc[u + 1].y * inv),
                                  pack_bf16x2(acc[u + 1].z * inv, acc[u + 1].w * inv));
@@ -775,8 +781,10 @@ cudaError_t init_umma_kernel() {
 
 int auto_attn_impl(const goose_ctx* c, int S, int B, int H) {
     (void)S; (void)H;
-    if (!c->encode_tiled) return GOOSE_ATTN_MMA;
-    return B >= 32 ? GOOSE_ATTN_UMMA : GOOSE_ATTN_MMA;
+    (void)B;
+    // the tcgen05 kernel wins at every tree size measured (B = 16: 15.8 us vs 31 us on the tiny workload);
+    // the mma.sync kernel remains as the path for drivers that cannot encode tensor maps and on request
+    return c->encode_tiled ? GOOSE_ATTN_UMMA : GOOSE_ATTN_MMA;
 }
 
 cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __nv_bfloat16* kc,
@@ -792,21 +800,14 @@ cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __
         return cudaErrorInvalidValue;
     int grid = c->num_sms;
     if (2 * grid > c->n_slots) grid = c->n_slots / 2;
-    tree_attn_umma_kernel<<<grid, kThreads, kUmmaSmem, st>>>(mq, mk, mv, row_off, ctx_len, parent, S, B, H,
-                                                            scale * kLog2e, c->partials, c->status,
-                                                            out, lse);
+    cudaError_t e = launch_pdl(tree_attn_umma_kernel, dim3(grid), dim3(kThreads), kUmmaSmem, st, mq, mk, mv, row_off,
+                               ctx_len, parent, S, B, H, scale * kLog2e, c->partials, c->status, out, lse);
     c->launches++;
-    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     dim3 cgrid((B + 31) / 32, H, S);
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = cgrid; cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = 0; cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
     const float* parts = c->partials;
-    e = cudaLaunchKernelEx(&cfg, tree_attn_combine_kernel, ctx_len, parent, S, B, H, grid, parts, out, lse);
+    e = launch_pdl(tree_attn_combine_kernel, cgrid, dim3(kCombineThreads), 0, st, ctx_len, parent, S, B, H, grid, parts,
+                   out, lse);
     c->launches++;
     return e;
 }

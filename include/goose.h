@@ -49,6 +49,7 @@ extern "C" {
 #define GOOSE_MAX_K      16   /* top-k width                                                       */
 #define GOOSE_HEAD_DIM  128   /* the only supported head dimension                                 */
 #define GOOSE_MAX_V  262144   /* vocabulary size limit of goose_node_topk                          */
+#define GOOSE_STATIC_TOPK_MAX_ROWS 2048   /* row limit of goose_node_topk_static                    */
 
 /* per-sequence status bits (goose_last_status) */
 #define GOOSE_ST_BAD_PARENT   1   /* parent[] is not a rooted tree in topological order */
@@ -100,6 +101,26 @@ int goose_tree_attn(goose_ctx* ctx, const void* q, const void* k_cache, const vo
  *   argmax int32 [rows]; topk_ids int32 [rows][k]; topk_vals fp32 [rows][k] (exact values) or NULL */
 int goose_node_topk(goose_ctx* ctx, const void* logits, int rows, int V, int64_t ldl, int k,
                     int32_t* argmax, int32_t* topk_ids, float* topk_vals, void* stream);
+
+/* goose_node_topk without a context and without any allocation.  (The paper has no counterpart: this
+ * entry point exists for integration reasons only.)
+ * Some hosts may not allocate device memory once they are running: an inference server that plans all
+ * of its device memory up front and treats a later cudaMalloc as an error, or a plug-in that is called
+ * at a point where entering the allocator (and the implicit device synchronisation it can cause) is not
+ * allowed.  goose_create allocates, so such callers cannot use goose_node_topk.  This variant computes
+ * exactly the same result with the same kernel; its only scratch (the per-chunk winners and arrival
+ * counters used when a row is longer than 32768 elements) is a fixed array of about 2 MiB that is part
+ * of the library image, so every GPU that loads the library holds it until the process exits.
+ *   - Arguments, layouts and results as goose_node_topk, all data pointers on the CURRENT device;
+ *     rows <= GOOSE_STATIC_TOPK_MAX_ROWS, otherwise GOOSE_EINVAL (nothing is enqueued).
+ *   - It calls no cudaMalloc / cudaFree and no allocating library routine.  The first call on each
+ *     device looks up the device address of the array (cudaGetSymbolAddress, with that device current);
+ *     make that first call outside any stream capture.
+ *   - All calls share the one array, which keeps the contents of the previous call; the counters it
+ *     needs at zero are cleared on `stream` before the kernel.  Two calls whose kernels may overlap on
+ *     the GPU (different streams, no dependency between them) race on the array: serialise them.      */
+int goose_node_topk_static(const void* logits, int rows, int V, int64_t ldl, int k,
+                           int32_t* argmax, int32_t* topk_ids, float* topk_vals, void* stream);
 
 /* Greedy acceptance walk (Algorithm 3, UnifiedGreedyWalk).  From node 0, repeatedly move to the
  * child c of the current node v with draft_tok[c] == argmax[v]; stop when no child matches.

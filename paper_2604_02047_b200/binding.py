@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libgoose.so")
 EXPORTS = [
     "goose_create", "goose_destroy", "goose_strerror", "goose_set_attn_impl", "goose_tree_attn",
     "goose_node_topk", "goose_accept", "goose_kv_compact", "goose_verify_step",
-    "goose_verify_step_host", "goose_last_status", "goose_launch_count",
+    "goose_verify_step_host", "goose_last_status", "goose_launch_count", "goose_node_topk_static",
 ]
 
 ATTN_AUTO, ATTN_MMA, ATTN_UMMA = 0, 1, 2
@@ -210,6 +210,23 @@ class Goose:
             _p(h_outs["topk_vals"]), _p(h_outs["path"]), _p(h_outs["accept_len"]), _p(h_outs["bonus"]),
             _p(h_outs["new_ctx_len"]), _stream()), "goose_verify_step_host")
         return h_outs
+
+
+def node_topk_static(logits: torch.Tensor, k: int, V: Optional[int] = None, want_vals: bool = True):
+    """``goose_node_topk_static``: top-k without a context and without any device allocation inside the
+    library (the output tensors are the caller's, allocated here by torch before the call)."""
+    lib = load_library()
+    _dev(logits, torch.bfloat16, "logits")
+    rows, ldl = logits.shape
+    V = ldl if V is None else V
+    argmax = torch.empty(rows, dtype=torch.int32, device=logits.device)
+    ids = torch.empty((rows, k), dtype=torch.int32, device=logits.device)
+    vals = torch.empty((rows, k), dtype=torch.float32, device=logits.device) if want_vals else None
+    with torch.cuda.device(logits.device):
+        _check(lib.goose_node_topk_static(_p(logits), ctypes.c_int(rows), ctypes.c_int(V), ctypes.c_int64(ldl),
+                                          ctypes.c_int(k), _p(argmax), _p(ids), _p(vals), _stream()),
+               "goose_node_topk_static")
+    return argmax, ids, vals
 
 
 # ---------------------------------------------------------------------- helpers for tests / bench

@@ -11,6 +11,8 @@
 // above T (a constant row) take an exact slow path over all keys.  Rows longer than one chunk
 // (V > 32768) finish with a merge of the chunks' candidates by the last CTA to arrive for the row
 // (arrival counter, no spinning).
+#include <mutex>
+
 #include "goose_internal.cuh"
 
 namespace goose {
@@ -283,4 +285,57 @@ cudaError_t launch_node_topk(goose_ctx* c, const __nv_bfloat16* logits, int rows
     return cudaSuccess;
 }
 
+
+// ---------------------------------------------------------------------------------------------------
+// goose_node_topk_static: the same kernel for callers that are not allowed to allocate device memory
+// (a host that pre-plans all device memory and forbids cudaMalloc at run time, or code running where
+// the allocator must not be entered).  The cross-chunk scratch lives in a file-scope device array that
+// every GPU loading this library carries until the process exits.
+constexpr int kStaticMaxRows = GOOSE_STATIC_TOPK_MAX_ROWS;
+constexpr size_t kStaticCandWords = (size_t)kStaticMaxRows * kTopkMaxChunks * kMaxK;   // per (row, chunk) winners: 2 MiB
+constexpr size_t kStaticCounterWords = kStaticMaxRows / 2;                             // int32 arrival counters: 8 KiB
+static __device__ __align__(256) u64 g_static_topk[kStaticCandWords + kStaticCounterWords];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+u64* g_static_ptr[kMaxDevices] = {};                             // device address of g_static_topk, per device
+}  // namespace
+
 }  // namespace goose
+
+extern "C" int goose_node_topk_static(const void* logits, int rows, int V, int64_t ldl, int k,
+                                      int32_t* argmax, int32_t* topk_ids, float* topk_vals, void* stream) {
+    using namespace goose;
+    if (!logits || !argmax || !topk_ids) return GOOSE_EINVAL;
+    if (rows < 0 || rows > kStaticMaxRows) return GOOSE_EINVAL;          // beyond the static scratch
+    if (V < 1 || V > GOOSE_MAX_V || ldl < V || (ldl & 7) != 0) return GOOSE_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(logits) & 15u) != 0) return GOOSE_EINVAL;
+    if (k < 1 || k > GOOSE_MAX_K || k > V) return GOOSE_EINVAL;
+    if (rows == 0) return GOOSE_OK;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return GOOSE_ECUDA;
+    u64* scratch;
+    {
+        // In host code the name g_static_topk is only a handle for the runtime, not a device address:
+        // resolve the address once per device, with that device current.
+        std::lock_guard<std::mutex> lock(g_static_mu);
+        if (!g_static_ptr[dev]) {
+            u64* p = nullptr;
+            if (cudaGetSymbolAddress((void**)&p, g_static_topk) != cudaSuccess || !p) return GOOSE_ECUDA;
+            g_static_ptr[dev] = p;
+        }
+        scratch = g_static_ptr[dev];
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int chunks = (V + kTopkChunk - 1) / kTopkChunk;
+    // the counters must start at zero; the array keeps whatever an earlier (possibly interrupted) call left
+    int32_t* counters = reinterpret_cast<int32_t*>(scratch + kStaticCandWords);
+    if (chunks > 1 && cudaMemsetAsync(counters, 0, sizeof(int32_t) * (size_t)rows, st) != cudaSuccess)
+        return GOOSE_ECUDA;
+    dim3 grid(chunks, rows);                                             // rows <= 2048 < 65535
+    cudaError_t e = launch_pdl(k <= 8 ? node_topk_kernel<8> : node_topk_kernel<16>, grid, dim3(kTopkThreads), 0, st,
+                               static_cast<const __nv_bfloat16*>(logits), V, ldl, k, chunks, scratch,
+                               counters, argmax, topk_ids, topk_vals);
+    return e == cudaSuccess ? GOOSE_OK : GOOSE_ECUDA;
+}

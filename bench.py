@@ -33,7 +33,7 @@ UNIT = "steps/s"
 L2_BYTES = 126 * 1024 * 1024
 # DRAM traffic per attention launch from the ncu capture summarised under profiles/ (bytes), per config
 # name; None = not captured for that workload.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"33b": 227_728_128}     # tree_attn_umma_kernel: 223.28 MB read + 4.44 MB written per launch
 
 
 def _peaks():

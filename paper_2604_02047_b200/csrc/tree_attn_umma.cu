@@ -22,6 +22,7 @@
 // Every wait in this file is bounded: when a wait runs out of polls the CTA raises an abort flag,
 // sets GOOSE_ST_TIMEOUT, drains its own copies in flight (again bounded), frees its TMEM and returns.
 #include <cuda.h>
+#include <cstdlib>
 
 #include "goose_internal.cuh"
 
@@ -43,7 +44,6 @@ constexpr uint32_t kColS = 0, kColO = 256;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;       // rescale O only when the running max grew by > 2^8
-constexpr int kCombineChunk = 8;                 // partials merged per pass of the combine kernel
 constexpr int kCombineThreads = 256;
 constexpr long long kWaitCycles = 2000000000ll;  // bound of every wait: about one second of SM clock
 
@@ -613,13 +613,16 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                     const int slot = 2 * blockIdx.x + (t_first == 0 ? 1 : 0);
                     float* part = partials + (size_t)slot * kPartialFloats;
                     if (row < B) {
+                        // invalid parent[]: a neutral partial (O = 0; the head's first part carries weight 1)
+                        // makes the combine kernel produce the defined zero output without re-validating
                         float4* dst = reinterpret_cast<float4*>(part) + row;
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
-                            dst[c * 128] = make_float4(__uint_as_float(v[4 * c]), __uint_as_float(v[4 * c + 1]),
-                                                       __uint_as_float(v[4 * c + 2]), __uint_as_float(v[4 * c + 3]));
-                        part[kMaxB * kHeadDim + row] = m_run;
-                        part[kMaxB * kHeadDim + kMaxB + row] = l_run;
+                            dst[c * 128] = bad ? make_float4(0.f, 0.f, 0.f, 0.f)
+                                               : make_float4(__uint_as_float(v[4 * c]), __uint_as_float(v[4 * c + 1]),
+                                                             __uint_as_float(v[4 * c + 2]), __uint_as_float(v[4 * c + 3]));
+                        part[kMaxB * kHeadDim + row] = bad ? (t_first == 0 ? 0.f : -INFINITY) : m_run;
+                        part[kMaxB * kHeadDim + kMaxB + row] = bad ? (t_first == 0 ? 1.f : 0.f) : l_run;
                     }
                     if (sm_tid == 0) TRACE(2, tn, 5);
                 }
@@ -645,10 +648,9 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
 //   M = max m_p,  L = sum l_p 2^(m_p - M),  out = sum_p 2^(m_p - M) O_p / L.
 // Lane <-> row (coalesced float4 loads of the transposed partial layout), warp <-> 16 output columns.
 __global__ void __launch_bounds__(kCombineThreads)
-tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ parent,
-                         int S, int B, int H, int G, const float* __restrict__ partials,
-                         __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
-    __shared__ int slot_s[kCombineChunk];
+tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, int S, int B, int H, int G,
+                         const float* __restrict__ partials, __nv_bfloat16* __restrict__ out,
+                         float* __restrict__ lse) {
     const int rg = blockIdx.x, h = blockIdx.y, s = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     pdl_wait();                                            // the main kernel's partials are complete and visible
@@ -665,88 +667,63 @@ tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, const int32_t* __r
     const long long head_first = off + (long long)h * T;
     const int c_lo = wk.cta_of(head_first), c_hi = wk.cta_of(head_first + T - 1);
     if (c_lo == c_hi) return;                              // written directly by the main kernel
-    // invalid parent[] -> zero-filled output (the main kernel has already set the status word)
-    int bad = 0;
-    for (int i = tid; i < B; i += kCombineThreads) {
-        int p = parent[(size_t)s * B + i];
-        bad |= (i == 0) ? (p != -1) : (p < 0 || p >= i);
-    }
-    bad = __syncthreads_or(bad);
     const int row = rg * 32 + lane;
-    const bool row_ok = row < B;
-    const int rr = row_ok ? row : 0;
+    if (row >= B) return;
+    // CTA c's partial for this head sits in slot 2c, or 2c+1 when its segment starts at the head's first tile,
+    // which only the first CTA can do.  With fewer items than CTAs some CTAs in [c_lo, c_hi] are empty.
+    const int flag_lo = wk.cta_start(c_lo) <= head_first ? 1 : 0;
+    const bool sparse = tot < G;
     float M_run = -INFINITY, L_run = 0.f;
     float4 acc[4];                                         // warp w owns column groups 4w .. 4w+3 (16 columns)
 #pragma unroll
     for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
 
-    // parts in chunks; a running (M, L) with rescaling of the accumulators keeps chunks independent
-    for (int cb = c_lo; cb <= c_hi; cb += kCombineChunk) {
-        __syncthreads();
-        if (tid < kCombineChunk) {
-            const int c = cb + tid;
-            int sl = -1;
-            if (c <= c_hi) {
-                const long long cs = wk.cta_start(c);
-                if (wk.cta_start(c + 1) > cs) sl = 2 * c + ((cs <= head_first) ? 1 : 0);
-            }
-            slot_s[tid] = sl;
-        }
-        __syncthreads();
-        float mp[kCombineChunk], lp[kCombineChunk];
+    // four parts per round: their (m, l) and their 4 x 16-byte accumulator pieces are loaded together
+    // (24 independent loads in flight per thread); a running (M, L) with rescaling merges the rounds
+    for (int cb = c_lo; cb <= c_hi; cb += 4) {
+        float mp[4], lp[4];
+        float4 x[4][4];
 #pragma unroll
-        for (int pi = 0; pi < kCombineChunk; ++pi) {
-            const int sl = slot_s[pi];
-            const float* pp = partials + (size_t)(sl < 0 ? 0 : sl) * kPartialFloats + kMaxB * kHeadDim;
-            const bool use = sl >= 0 && row_ok;
-            mp[pi] = use ? __ldcg(pp + row) : -INFINITY;
-            lp[pi] = use ? __ldcg(pp + kMaxB + row) : 0.f;
+        for (int q = 0; q < 4; ++q) {
+            const int c = cb + q;
+            bool use = c <= c_hi;
+            if (use && sparse) use = wk.cta_start(c + 1) > wk.cta_start(c);
+            const int sl = use ? 2 * c + (c == c_lo ? flag_lo : 0) : 0;
+            const float* pp = partials + (size_t)sl * kPartialFloats;
+            mp[q] = use ? __ldcg(pp + kMaxB * kHeadDim + row) : -INFINITY;
+            lp[q] = use ? __ldcg(pp + kMaxB * kHeadDim + kMaxB + row) : 0.f;
+            const float4* p4 = reinterpret_cast<const float4*>(pp) + row;
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                x[q][u] = use ? __ldcg(p4 + (4 * warp + u) * 128) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
         float M_new = M_run;
 #pragma unroll
-        for (int pi = 0; pi < kCombineChunk; ++pi) M_new = fmaxf(M_new, mp[pi]);
+        for (int q = 0; q < 4; ++q) M_new = fmaxf(M_new, mp[q]);
         const float a_old = (M_run == -INFINITY) ? 0.f : ex2(M_run - M_new);
         L_run *= a_old;
 #pragma unroll
         for (int u = 0; u < 4; ++u) { acc[u].x *= a_old; acc[u].y *= a_old; acc[u].z *= a_old; acc[u].w *= a_old; }
 #pragma unroll
-        for (int pi = 0; pi < kCombineChunk; ++pi) {
-            const float w = (mp[pi] == -INFINITY) ? 0.f : ex2(mp[pi] - M_new);
-            L_run += w * lp[pi];
-            mp[pi] = w;                                    // from here on: the part's weight for this row
+        for (int q = 0; q < 4; ++q) {
+            const float w = (mp[q] == -INFINITY) ? 0.f : ex2(mp[q] - M_new);
+            L_run += w * lp[q];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                acc[u].x += w * x[q][u].x; acc[u].y += w * x[q][u].y;
+                acc[u].z += w * x[q][u].z; acc[u].w += w * x[q][u].w;
+            }
         }
         M_run = M_new;
-#pragma unroll
-        for (int p0 = 0; p0 < kCombineChunk; p0 += 4) {    // four parts = 16 independent 16-byte loads in flight
-            if (slot_s[p0] < 0 && slot_s[p0 + 1] < 0 && slot_s[p0 + 2] < 0 && slot_s[p0 + 3] < 0) continue;
-            float4 x[4][4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int sl = slot_s[p0 + q];
-                const float4* pp = reinterpret_cast<const float4*>(partials + (size_t)(sl < 0 ? 0 : sl) * kPartialFloats) + rr;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) x[q][u] = __ldcg(pp + (4 * warp + u) * 128);
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const float w = slot_s[p0 + q] < 0 ? 0.f : mp[p0 + q];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    acc[u].x += w * x[q][u].x; acc[u].y += w * x[q][u].y;
-                    acc[u].z += w * x[q][u].z; acc[u].w += w * x[q][u].w;
-                }
-            }
-        }
     }
-    if (!row_ok) return;
-    const float inv = bad ? 0.f : 1.f / L_run;
+    const float inv = 1.f / L_run;
     uint4* dst = reinterpret_cast<uint4*>(out + (((size_t)s * B + row) * H + h) * kHeadDim + 16 * warp);
 #pragma unroll
     for (int u = 0; u < 4; u += 2)
         dst[u >> 1] = make_uint4(pack_bf16x2(acc[u].x * inv, acc[u].y * inv), pack_bf16x2(acc[u].z * inv, acc[u].w * inv),
                                  pack_bf16x2(acc[u + 1].x * inv, acc[u + 1].y * inv),
                                  pack_bf16x2(acc[u + 1].z * inv, acc[u + 1].w * inv));
-    if (lse && warp == 0) lse[((size_t)s * B + row) * H + h] = bad ? 0.f : (M_run + log2f(L_run)) * kLn2;
+    if (lse && warp == 0) lse[((size_t)s * B + row) * H + h] = (M_run + log2f(L_run)) * kLn2;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -804,10 +781,12 @@ cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __
                                ctx_len, parent, S, B, H, scale * kLog2e, c->partials, c->status, out, lse);
     c->launches++;
     if (e != cudaSuccess) return e;
+#ifdef GOOSE_TRACE
+    if (getenv("GOOSE_SKIP_COMBINE")) return e;       // debug build only: time the main kernel alone
+#endif
     dim3 cgrid((B + 31) / 32, H, S);
     const float* parts = c->partials;
-    e = launch_pdl(tree_attn_combine_kernel, cgrid, dim3(kCombineThreads), 0, st, ctx_len, parent, S, B, H, grid, parts,
-                   out, lse);
+    e = launch_pdl(tree_attn_combine_kernel, cgrid, dim3(kCombineThreads), 0, st, ctx_len, S, B, H, grid, parts, out, lse);
     c->launches++;
     return e;
 }

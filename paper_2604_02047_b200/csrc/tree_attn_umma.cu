@@ -22,6 +22,7 @@
 // Every wait in this file is bounded: when a wait runs out of polls the CTA raises an abort flag,
 // sets GOOSE_ST_TIMEOUT, drains its own copies in flight (again bounded), frees its TMEM and returns.
 #include <cuda.h>
+#include <cuda_fp16.h>
 #include <cstdlib>
 
 #include "goose_internal.cuh"
@@ -45,6 +46,10 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;       // rescale O only when the running max grew by > 2^8
 constexpr int kCombineThreads = 256;
+// split-KV partial of this kernel: normalised O/l as fp16, uint4 [16 column groups of 8][128 rows] (32 KB, a warp's
+// stores and the combine kernel's loads are contiguous), then m[128], l[128] as fp32
+constexpr int kPartHalfWords = 16 * 128 * 4;     // 32-bit words of the fp16 block
+constexpr int kUmmaPartFloats = kPartHalfWords + 2 * kMaxB;
 constexpr long long kWaitCycles = 2000000000ll;  // bound of every wait: about one second of SM clock
 
 #ifdef GOOSE_TRACE
@@ -282,6 +287,12 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = hd->tmem_base;
+    // L2 prefetch hints for the small index arrays (a hint reads no data, so it may precede the wait)
+    if (threadIdx.x == 32) {
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(ctx_len));
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(row_off));
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(parent));
+    }
     // everything above touched no global memory: now wait for the preceding kernel, then let the next
     // one (the combine kernel) get resident early -- it waits for this grid before reading the partials
     pdl_wait();
@@ -607,22 +618,28 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                         if (lse) lse[((size_t)s0 * B + row) * H + h0] = bad ? 0.f : (m_run + log2f(l_run)) * kLn2;
                     }
                 } else {
-                    // partial -> workspace slot of this CTA (combined by tree_attn_combine_kernel).
-                    // Layout: float4 [32 column groups][128 rows] so that a warp's stores (and the
-                    // combine kernel's loads) are contiguous, then m[128], l[128].
+                    // partial -> workspace slot of this CTA (combined by tree_attn_combine_kernel): O/l in fp16
+                    // (relative error 2^-11, far below the bf16 rounding of the final output), m and l in fp32
                     const int slot = 2 * blockIdx.x + (t_first == 0 ? 1 : 0);
-                    float* part = partials + (size_t)slot * kPartialFloats;
+                    float* part = partials + (size_t)slot * kUmmaPartFloats;
                     if (row < B) {
                         // invalid parent[]: a neutral partial (O = 0; the head's first part carries weight 1)
                         // makes the combine kernel produce the defined zero output without re-validating
-                        float4* dst = reinterpret_cast<float4*>(part) + row;
+                        const float inv = (bad || l_run == 0.f) ? 0.f : 1.f / l_run;
+                        uint4* dst = reinterpret_cast<uint4*>(part) + row;
 #pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            dst[c * 128] = bad ? make_float4(0.f, 0.f, 0.f, 0.f)
-                                               : make_float4(__uint_as_float(v[4 * c]), __uint_as_float(v[4 * c + 1]),
-                                                             __uint_as_float(v[4 * c + 2]), __uint_as_float(v[4 * c + 3]));
-                        part[kMaxB * kHeadDim + row] = bad ? (t_first == 0 ? 0.f : -INFINITY) : m_run;
-                        part[kMaxB * kHeadDim + kMaxB + row] = bad ? (t_first == 0 ? 1.f : 0.f) : l_run;
+                        for (int c = 0; c < 16; ++c) {
+                            uint32_t hw[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                __half2 h2 = __floats2half2_rn(__uint_as_float(v[8 * c + 2 * e]) * inv,
+                                                               __uint_as_float(v[8 * c + 2 * e + 1]) * inv);
+                                hw[e] = *reinterpret_cast<uint32_t*>(&h2);
+                            }
+                            dst[c * 128] = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                        }
+                        part[kPartHalfWords + row] = bad ? (t_first == 0 ? 0.f : -INFINITY) : m_run;
+                        part[kPartHalfWords + kMaxB + row] = bad ? (t_first == 0 ? 1.f : 0.f) : l_run;
                     }
                     if (sm_tid == 0) TRACE(2, tn, 5);
                 }
@@ -674,28 +691,28 @@ tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, int S, int B, int 
     const int flag_lo = wk.cta_start(c_lo) <= head_first ? 1 : 0;
     const bool sparse = tot < G;
     float M_run = -INFINITY, L_run = 0.f;
-    float4 acc[4];                                         // warp w owns column groups 4w .. 4w+3 (16 columns)
+    float acc[16];                                         // warp w owns columns 16w .. 16w+15 (column groups 2w, 2w+1)
 #pragma unroll
-    for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int u = 0; u < 16; ++u) acc[u] = 0.f;
 
-    // four parts per round: their (m, l) and their 4 x 16-byte accumulator pieces are loaded together
-    // (24 independent loads in flight per thread); a running (M, L) with rescaling merges the rounds
+    // four parts per round: their (m, l) and their two 16-byte pieces of O/l are loaded together
+    // (16 independent loads in flight per thread); a running (M, L) with rescaling merges the rounds
     for (int cb = c_lo; cb <= c_hi; cb += 4) {
         float mp[4], lp[4];
-        float4 x[4][4];
+        uint4 x[4][2];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             const int c = cb + q;
             bool use = c <= c_hi;
             if (use && sparse) use = wk.cta_start(c + 1) > wk.cta_start(c);
             const int sl = use ? 2 * c + (c == c_lo ? flag_lo : 0) : 0;
-            const float* pp = partials + (size_t)sl * kPartialFloats;
-            mp[q] = use ? __ldcg(pp + kMaxB * kHeadDim + row) : -INFINITY;
-            lp[q] = use ? __ldcg(pp + kMaxB * kHeadDim + kMaxB + row) : 0.f;
-            const float4* p4 = reinterpret_cast<const float4*>(pp) + row;
+            const float* pp = partials + (size_t)sl * kUmmaPartFloats;
+            mp[q] = use ? __ldcg(pp + kPartHalfWords + row) : -INFINITY;
+            lp[q] = use ? __ldcg(pp + kPartHalfWords + kMaxB + row) : 0.f;
+            const uint4* p4 = reinterpret_cast<const uint4*>(pp) + row;
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-                x[q][u] = use ? __ldcg(p4 + (4 * warp + u) * 128) : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int u = 0; u < 2; ++u)
+                x[q][u] = use ? __ldcg(p4 + (2 * warp + u) * 128) : make_uint4(0u, 0u, 0u, 0u);
         }
         float M_new = M_run;
 #pragma unroll
@@ -703,15 +720,20 @@ tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, int S, int B, int 
         const float a_old = (M_run == -INFINITY) ? 0.f : ex2(M_run - M_new);
         L_run *= a_old;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) { acc[u].x *= a_old; acc[u].y *= a_old; acc[u].z *= a_old; acc[u].w *= a_old; }
+        for (int u = 0; u < 16; ++u) acc[u] *= a_old;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            const float w = (mp[q] == -INFINITY) ? 0.f : ex2(mp[q] - M_new);
-            L_run += w * lp[q];
+            const float w = ((mp[q] == -INFINITY) ? 0.f : ex2(mp[q] - M_new)) * lp[q];   // un-normalise: O_p = x_p * l_p
+            L_run += w;
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                acc[u].x += w * x[q][u].x; acc[u].y += w * x[q][u].y;
-                acc[u].z += w * x[q][u].z; acc[u].w += w * x[q][u].w;
+            for (int u = 0; u < 2; ++u) {
+                const uint32_t hw[4] = {x[q][u].x, x[q][u].y, x[q][u].z, x[q][u].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&hw[e]));
+                    acc[8 * u + 2 * e] += w * f.x;
+                    acc[8 * u + 2 * e + 1] += w * f.y;
+                }
             }
         }
         M_run = M_new;
@@ -719,10 +741,9 @@ tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, int S, int B, int 
     const float inv = 1.f / L_run;
     uint4* dst = reinterpret_cast<uint4*>(out + (((size_t)s * B + row) * H + h) * kHeadDim + 16 * warp);
 #pragma unroll
-    for (int u = 0; u < 4; u += 2)
-        dst[u >> 1] = make_uint4(pack_bf16x2(acc[u].x * inv, acc[u].y * inv), pack_bf16x2(acc[u].z * inv, acc[u].w * inv),
-                                 pack_bf16x2(acc[u + 1].x * inv, acc[u + 1].y * inv),
-                                 pack_bf16x2(acc[u + 1].z * inv, acc[u + 1].w * inv));
+    for (int u = 0; u < 2; ++u)
+        dst[u] = make_uint4(pack_bf16x2(acc[8 * u] * inv, acc[8 * u + 1] * inv), pack_bf16x2(acc[8 * u + 2] * inv, acc[8 * u + 3] * inv),
+                            pack_bf16x2(acc[8 * u + 4] * inv, acc[8 * u + 5] * inv), pack_bf16x2(acc[8 * u + 6] * inv, acc[8 * u + 7] * inv));
     if (lse && warp == 0) lse[((size_t)s * B + row) * H + h] = (M_run + log2f(L_run)) * kLn2;
 }
 

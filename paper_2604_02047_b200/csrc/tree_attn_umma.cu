@@ -46,6 +46,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;       // rescale O only when the running max grew by > 2^8
 constexpr int kCombineThreads = 256;
+constexpr int kCombineRound = 4;                 // partials merged per load round of the combine kernel
 // split-KV partial of this kernel: normalised O/l as fp16, uint4 [16 column groups of 8][128 rows] (32 KB, a warp's
 // stores and the combine kernel's loads are contiguous), then m[128], l[128] as fp32
 constexpr int kPartHalfWords = 16 * 128 * 4;     // 32-bit words of the fp16 block
@@ -213,10 +214,20 @@ struct Work {
     const int32_t* ctx_len;
     int S, H, B, G;
     long long total;          // all items
+    bool small;               // total * (G + 1) fits 31 bits: 32-bit arithmetic (64-bit division is slow on the GPU)
     __device__ __forceinline__ int tiles(int s) const { return (ctx_len[s] + B + kTile - 1) / kTile; }
-    __device__ __forceinline__ long long cta_start(int c) const { return total * c / G; }
+    __device__ __forceinline__ void init() {
+        long long tot = 0;
+        for (int s = 0; s < S; ++s) tot += (long long)H * tiles(s);
+        total = tot;
+        small = tot * (G + 1) < 0x7FFFFFFFll;
+    }
+    __device__ __forceinline__ long long cta_start(int c) const {
+        if (small) return ((uint32_t)total * (uint32_t)c) / (uint32_t)G;
+        return total * c / G;
+    }
     __device__ __forceinline__ int cta_of(long long w) const {
-        int c = (int)(w * G / total);
+        int c = small ? (int)(((uint32_t)w * (uint32_t)G) / (uint32_t)total) : (int)(w * G / total);
         if (c >= G) c = G - 1;
         while (c + 1 < G && cta_start(c + 1) <= w) ++c;
         while (c > 0 && cta_start(c) > w) --c;
@@ -237,8 +248,9 @@ struct Cursor {               // walks items in order
             TT = wk.tiles(ss);
         }
         s = ss; T = TT; w = w0;
-        h = (int)((w0 - off) / TT);
-        t = (int)((w0 - off) % TT);
+        const long long rem = w0 - off;
+        h = wk.small ? (int)((uint32_t)rem / (uint32_t)TT) : (int)(rem / TT);
+        t = (int)(rem - (long long)h * TT);
     }
     __device__ __forceinline__ void next(const Work& wk) {
         ++w; ++t;
@@ -299,11 +311,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     pdl_trigger();
     Work wk;
     wk.ctx_len = ctx_len; wk.S = S; wk.H = H; wk.B = B; wk.G = gridDim.x;
-    {
-        long long tot = 0;
-        for (int s = 0; s < S; ++s) tot += (long long)H * wk.tiles(s);
-        wk.total = tot;
-    }
+    wk.init();
     const long long w_begin = wk.cta_start(blockIdx.x), w_end = wk.cta_start(blockIdx.x + 1);
 
 
@@ -674,12 +682,9 @@ tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, int S, int B, int 
     pdl_trigger();
     Work wk;
     wk.ctx_len = ctx_len; wk.S = S; wk.H = H; wk.B = B; wk.G = G;
-    long long tot = 0, off = 0;
-    for (int ss = 0; ss < S; ++ss) {
-        if (ss == s) off = tot;
-        tot += (long long)H * wk.tiles(ss);
-    }
-    wk.total = tot;
+    wk.init();
+    long long off = 0;
+    for (int ss = 0; ss < s; ++ss) off += (long long)H * wk.tiles(ss);
     const int T = wk.tiles(s);
     const long long head_first = off + (long long)h * T;
     const int c_lo = wk.cta_of(head_first), c_hi = wk.cta_of(head_first + T - 1);
@@ -689,19 +694,19 @@ tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, int S, int B, int 
     // CTA c's partial for this head sits in slot 2c, or 2c+1 when its segment starts at the head's first tile,
     // which only the first CTA can do.  With fewer items than CTAs some CTAs in [c_lo, c_hi] are empty.
     const int flag_lo = wk.cta_start(c_lo) <= head_first ? 1 : 0;
-    const bool sparse = tot < G;
+    const bool sparse = wk.total < G;
     float M_run = -INFINITY, L_run = 0.f;
     float acc[16];                                         // warp w owns columns 16w .. 16w+15 (column groups 2w, 2w+1)
 #pragma unroll
     for (int u = 0; u < 16; ++u) acc[u] = 0.f;
 
-    // four parts per round: their (m, l) and their two 16-byte pieces of O/l are loaded together
+    // kCombineRound parts per round: their (m, l) and their two 16-byte pieces of O/l are loaded together
     // (16 independent loads in flight per thread); a running (M, L) with rescaling merges the rounds
-    for (int cb = c_lo; cb <= c_hi; cb += 4) {
-        float mp[4], lp[4];
-        uint4 x[4][2];
+    for (int cb = c_lo; cb <= c_hi; cb += kCombineRound) {
+        float mp[kCombineRound], lp[kCombineRound];
+        uint4 x[kCombineRound][2];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int q = 0; q < kCombineRound; ++q) {
             const int c = cb + q;
             bool use = c <= c_hi;
             if (use && sparse) use = wk.cta_start(c + 1) > wk.cta_start(c);
@@ -716,13 +721,13 @@ tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, int S, int B, int 
         }
         float M_new = M_run;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) M_new = fmaxf(M_new, mp[q]);
+        for (int q = 0; q < kCombineRound; ++q) M_new = fmaxf(M_new, mp[q]);
         const float a_old = (M_run == -INFINITY) ? 0.f : ex2(M_run - M_new);
         L_run *= a_old;
 #pragma unroll
         for (int u = 0; u < 16; ++u) acc[u] *= a_old;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int q = 0; q < kCombineRound; ++q) {
             const float w = ((mp[q] == -INFINITY) ? 0.f : ex2(mp[q] - M_new)) * lp[q];   // un-normalise: O_p = x_p * l_p
             L_run += w;
 #pragma unroll

@@ -44,7 +44,7 @@ def lib() -> ctypes.CDLL:
         _lib = ctypes.CDLL(_LIB)
         _lib.oracle_num_threads.restype = ctypes.c_int
         for name in ("oracle_tree_attn", "oracle_tree_attn_rows", "oracle_node_topk", "oracle_accept",
-                     "oracle_kv_compact", "oracle_check_parent"):
+                     "oracle_kv_compact", "oracle_check_parent", "oracle_harvest"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
 
@@ -160,3 +160,22 @@ def kv_compact(k_cache, v_cache, row_off, ctx_len, path, accept_len
 def check_parent(parent) -> bool:
     parent = _c(parent, np.int32).reshape(-1)
     return lib().oracle_check_parent(_ptr(parent, ctypes.c_int32), ctypes.c_int(len(parent))) == 0
+
+
+def harvest(logits, k: int, row_tok, adj_ids: np.ndarray, adj_scores: np.ndarray, V: Optional[int] = None
+            ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """Harvest every logits row into the Tier-1 adjacency table (ids int32 [table_rows][k], scores fp64
+    [table_rows][k], both updated on copies).  Returns (adj_ids, adj_scores, row_lse)."""
+    logits = _c(logits, np.uint16)
+    rows, ldl = logits.shape
+    V = ldl if V is None else V
+    row_tok = _c(row_tok, np.int32).reshape(rows)
+    ids = np.ascontiguousarray(adj_ids, dtype=np.int32).copy()
+    sc = np.ascontiguousarray(adj_scores, dtype=np.float64).copy()
+    lse = np.zeros(rows, dtype=np.float64)
+    rc = lib().oracle_harvest(_ptr(logits, ctypes.c_uint16), ctypes.c_int(rows), ctypes.c_int(V), ctypes.c_int64(ldl),
+                              ctypes.c_int(k), _ptr(row_tok, ctypes.c_int32), ctypes.c_int(ids.shape[0]),
+                              _ptr(ids, ctypes.c_int32), _ptr(sc, ctypes.c_double), _ptr(lse, ctypes.c_double))
+    if rc != 0:
+        raise ValueError("oracle_harvest failed: rc=%d" % rc)
+    return ids, sc, lse

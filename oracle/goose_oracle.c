@@ -258,3 +258,39 @@ int oracle_kv_compact(const uint16_t* kc, const uint16_t* vc, const int64_t* row
     }
     return 0;
 }
+
+/* ------------------------------------------------------------------ logit harvest into the Tier-1 adjacency table
+ * App. "Aggressive logit harvesting" + "Dense GPU bigram adjacency table" (Tier 1, unigram): two dense
+ * [table_rows][k] tensors hold, for every vocabulary token, the ids and the "logit-derived scores" of its
+ * top-k successors; every row of every forward's logits is harvested, rejected branches included.
+ * Reading used here: row r of the logits predicts the successor of token row_tok[r]; its score is the softmax
+ * probability exp(logit - lse_r), lse_r = log sum_j exp(logit_j) over the first V entries.  Rows are harvested in
+ * order r = 0 .. rows-1, so when several rows carry the same token the LAST one is what the table keeps.
+ * Rows whose token is outside [0, table_rows) are skipped.  row_lse [rows] may be NULL. */
+int oracle_harvest(const uint16_t* logits, int rows, int V, int64_t ldl, int k, const int32_t* row_tok,
+                   int table_rows, int32_t* adj_ids, double* adj_scores, double* row_lse) {
+    if (k < 1 || k > V) return -1;
+    vi_t* a = (vi_t*)malloc(sizeof(vi_t) * (size_t)V);
+    if (!a) return -2;
+    for (int r = 0; r < rows; ++r) {
+        double mx = -INFINITY;
+        for (int j = 0; j < V; ++j) {
+            a[j].v = bf16_to_f64(logits[(size_t)r * ldl + j]);
+            a[j].idx = j;
+            if (a[j].v > mx) mx = a[j].v;
+        }
+        double sum = 0.0;
+        for (int j = 0; j < V; ++j) sum += exp(a[j].v - mx);
+        const double lse = mx + log(sum);
+        if (row_lse) row_lse[r] = lse;
+        const int tok = row_tok[r];
+        if (tok < 0 || tok >= table_rows) continue;
+        qsort(a, (size_t)V, sizeof(vi_t), cmp_vi);
+        for (int j = 0; j < k; ++j) {
+            adj_ids[(size_t)tok * k + j] = a[j].idx;
+            adj_scores[(size_t)tok * k + j] = exp(a[j].v - lse);
+        }
+    }
+    free(a);
+    return 0;
+}

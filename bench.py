@@ -217,6 +217,13 @@ def run_ours(args, x, cfg, rank, world, local_rank):
         d = reps[i % R]
         g.node_topk(d["logits"], x.k)
 
+    adj_ids = torch.full((x.V, x.k), -1, dtype=torch.int32, device=dev)
+    adj_scores = torch.zeros((x.V, x.k), dtype=torch.float32, device=dev)
+
+    def harvest(i):          # adjacent row of the path (not part of the step metric): top-k + lse + table scatter
+        d = reps[i % R]
+        g.harvest(d["logits"], x.k, d["draft_tok"].view(-1), adj_ids, adj_scores)
+
     with torch.cuda.stream(stream):
         for i in range(max(3, args.warmup)):
             step(i)
@@ -232,6 +239,7 @@ def run_ours(args, x, cfg, rank, world, local_rank):
         g_step, launches_per_step = capture(step)
         g_attn, _ = capture(attn)
         g_topk, _ = capture(topk)
+        g_harv, _ = capture(harvest)
 
         def time_graph(gr, rounds):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -266,6 +274,8 @@ def run_ours(args, x, cfg, rank, world, local_rank):
             attn_ms = time_graph(g_attn, attn_rounds) / (attn_rounds * R)
             time_graph(g_topk, 1)
             topk_ms = time_graph(g_topk, attn_rounds) / (attn_rounds * R)
+            time_graph(g_harv, 1)
+            harv_ms = time_graph(g_harv, attn_rounds) / (attn_rounds * R)
         clocks = clk.summary()
     value, ms_per_step = aggregate_steps_per_s(args.steps, local_ms, world, dev)
 
@@ -324,7 +334,7 @@ def run_ours(args, x, cfg, rank, world, local_rank):
                      "frac": attn_gbs / peak, "peak_kind": peak_kind,
                      "traffic": NCU_TRAFFIC_BYTES.get(cfg.name), "algorithmic_bytes": ab["attn"],
                      "us_per_launch": attn_ms * 1e3},
-        "kernels": {"tree_attn_us": attn_ms * 1e3, "node_topk_us": topk_ms * 1e3,
+        "kernels": {"tree_attn_us": attn_ms * 1e3, "node_topk_us": topk_ms * 1e3, "harvest_us": harv_ms * 1e3,
                     "node_topk_gbs": ab["topk"] / (topk_ms * 1e-3) / 1e9,
                     "step_gbs": ab["total"] / (ms_per_step * 1e-3) / 1e9,
                     "step_frac_of_peak": ab["total"] / (ms_per_step * 1e-3) / 1e9 / peak},

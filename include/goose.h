@@ -102,6 +102,21 @@ int goose_tree_attn(goose_ctx* ctx, const void* q, const void* k_cache, const vo
 int goose_node_topk(goose_ctx* ctx, const void* logits, int rows, int V, int64_t ldl, int k,
                     int32_t* argmax, int32_t* topk_ids, float* topk_vals, void* stream);
 
+/* Harvest of a forward's logits into the Tier-1 (unigram) adjacency table (App. C.1 "Aggressive logit
+ * harvesting"; "Dense GPU bigram adjacency table", Tier 1: two dense |V| x K tensors with the ids and the
+ * "logit-derived scores" of each token's top-K successors; every row is harvested, rejected branches and
+ * prefill rows included).  Runs goose_node_topk with the row log-sum-exp, then for every row r writes
+ *   adj_ids[row_tok[r]][j] = topk_ids[r][j],  adj_scores[row_tok[r]][j] = exp(topk_vals[r][j] - row_lse[r])
+ * i.e. the softmax probability of the successor.  Rows are harvested in row order: of several rows with
+ * the same token the last one is kept.  Rows whose token is outside [0, table_rows) are skipped; table
+ * rows of tokens that do not occur keep their contents.
+ *   row_tok int32 [rows]: the token whose successors row r predicts (a tree node's own draft token)
+ *   adj_ids int32 [table_rows][k], adj_scores fp32 [table_rows][k]   (updated in place)
+ *   argmax [rows], topk_ids [rows][k], topk_vals [rows][k], row_lse fp32 [rows]: outputs, all required       */
+int goose_harvest(goose_ctx* ctx, const void* logits, int rows, int V, int64_t ldl, int k, const int32_t* row_tok,
+                  int table_rows, int32_t* adj_ids, float* adj_scores, int32_t* argmax, int32_t* topk_ids,
+                  float* topk_vals, float* row_lse, void* stream);
+
 /* goose_node_topk without a context and without any allocation.  (The paper has no counterpart: this
  * entry point exists for integration reasons only.)
  * Some hosts may not allocate device memory once they are running: an inference server that plans all

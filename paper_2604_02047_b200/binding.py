@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libgoose.so")
 EXPORTS = [
     "goose_create", "goose_destroy", "goose_strerror", "goose_set_attn_impl", "goose_tree_attn",
     "goose_node_topk", "goose_accept", "goose_kv_compact", "goose_verify_step",
-    "goose_verify_step_host", "goose_last_status", "goose_launch_count", "goose_node_topk_static",
+    "goose_verify_step_host", "goose_last_status", "goose_launch_count", "goose_node_topk_static", "goose_harvest",
 ]
 
 ATTN_AUTO, ATTN_MMA, ATTN_UMMA = 0, 1, 2
@@ -141,6 +141,23 @@ class Goose:
         _check(self.lib.goose_node_topk(self.h, _p(logits), ctypes.c_int(rows), ctypes.c_int(V), ctypes.c_int64(ldl),
                                         ctypes.c_int(k), _p(argmax), _p(ids), _p(vals), _stream()), "goose_node_topk")
         return argmax, ids, vals
+
+    def harvest(self, logits, k: int, row_tok, adj_ids, adj_scores, V: Optional[int] = None):
+        """Top-k + log-sum-exp of every row, then scatter into the adjacency table (updated in place)."""
+        _dev(logits, torch.bfloat16, "logits"); _dev(row_tok, torch.int32, "row_tok")
+        _dev(adj_ids, torch.int32, "adj_ids"); _dev(adj_scores, torch.float32, "adj_scores")
+        rows, ldl = logits.shape
+        V = ldl if V is None else V
+        dev = logits.device
+        argmax = torch.empty(rows, dtype=torch.int32, device=dev)
+        ids = torch.empty((rows, k), dtype=torch.int32, device=dev)
+        vals = torch.empty((rows, k), dtype=torch.float32, device=dev)
+        lse = torch.empty(rows, dtype=torch.float32, device=dev)
+        _check(self.lib.goose_harvest(self.h, _p(logits), ctypes.c_int(rows), ctypes.c_int(V), ctypes.c_int64(ldl),
+                                      ctypes.c_int(k), _p(row_tok), ctypes.c_int(adj_ids.shape[0]), _p(adj_ids),
+                                      _p(adj_scores), _p(argmax), _p(ids), _p(vals), _p(lse), _stream()),
+               "goose_harvest")
+        return argmax, ids, vals, lse
 
     def accept(self, draft_tok, parent, argmax):
         _dev(draft_tok, torch.int32, "draft_tok"); _dev(parent, torch.int32, "parent"); _dev(argmax, torch.int32, "argmax")

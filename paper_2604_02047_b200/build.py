@@ -10,7 +10,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libgoose.so")
-SOURCES = ["api.cu", "node_topk.cu", "accept.cu", "kv_compact.cu", "tree_attn_mma.cu", "tree_attn_umma.cu"]
+SOURCES = ["api.cu", "node_topk.cu", "harvest.cu", "accept.cu", "kv_compact.cu", "tree_attn_mma.cu",
+           "tree_attn_umma.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
               "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
 

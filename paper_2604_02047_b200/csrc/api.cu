@@ -85,6 +85,7 @@ int goose_create(goose_ctx** out, int device, int max_S, int max_B, int max_H, i
     ok = ok && cudaMalloc(&c->head_counters, sizeof(int32_t) * (size_t)heads) == cudaSuccess;
     ok = ok && cudaMalloc(&c->topk_cand, sizeof(unsigned long long) * (size_t)c->topk_cand_cap) == cudaSuccess;
     ok = ok && cudaMalloc(&c->row_counters, sizeof(int32_t) * (size_t)c->topk_rows_cap) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->topk_lse_ws, sizeof(float) * 2 * (size_t)c->topk_rows_cap * kTopkMaxChunks) == cudaSuccess;
     ok = ok && cudaMalloc(&c->status, sizeof(int32_t) * (size_t)max_S) == cudaSuccess;
     if (ok) {
         ok = ok && cudaMemset(c->head_counters, 0, sizeof(int32_t) * (size_t)heads) == cudaSuccess;
@@ -112,7 +113,7 @@ int goose_destroy(goose_ctx* c) {
     if (!c) return GOOSE_EINVAL;
     cudaSetDevice(c->device);
     cudaFree(c->partials); cudaFree(c->head_counters); cudaFree(c->topk_cand);
-    cudaFree(c->row_counters); cudaFree(c->status); cudaFree(c->stage);
+    cudaFree(c->row_counters); cudaFree(c->topk_lse_ws); cudaFree(c->status); cudaFree(c->stage);
     delete c;
     return GOOSE_OK;
 }
@@ -158,7 +159,25 @@ int goose_node_topk(goose_ctx* c, const void* logits, int rows, int V, int64_t l
     if (V < 1 || V > GOOSE_MAX_V || ldl < V || (ldl & 7) != 0 || !aligned16(logits)) return GOOSE_EINVAL;
     if (k < 1 || k > GOOSE_MAX_K || k > V) return GOOSE_EINVAL;
     cudaError_t e = goose::launch_node_topk(c, (const __nv_bfloat16*)logits, rows, V, ldl, k, argmax, topk_ids,
-                                            topk_vals, static_cast<cudaStream_t>(stream));
+                                            topk_vals, nullptr, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e);
+    return GOOSE_OK;
+}
+
+int goose_harvest(goose_ctx* c, const void* logits, int rows, int V, int64_t ldl, int k, const int32_t* row_tok,
+                  int table_rows, int32_t* adj_ids, float* adj_scores, int32_t* argmax, int32_t* topk_ids,
+                  float* topk_vals, float* row_lse, void* stream) {
+    if (!c || !logits || !row_tok || !adj_ids || !adj_scores || !argmax || !topk_ids || !topk_vals || !row_lse)
+        return GOOSE_EINVAL;
+    if (rows < 0 || rows > c->topk_rows_cap || table_rows < 1) return GOOSE_EINVAL;
+    if (V < 1 || V > GOOSE_MAX_V || ldl < V || (ldl & 7) != 0 || !aligned16(logits)) return GOOSE_EINVAL;
+    if (k < 1 || k > GOOSE_MAX_K || k > V) return GOOSE_EINVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = goose::launch_node_topk(c, (const __nv_bfloat16*)logits, rows, V, ldl, k, argmax, topk_ids,
+                                            topk_vals, row_lse, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = goose::launch_harvest_scatter(c, row_tok, rows, table_rows, k, topk_ids, topk_vals, row_lse, adj_ids,
+                                      adj_scores, st);
     if (e != cudaSuccess) return cuda_fail(e);
     return GOOSE_OK;
 }

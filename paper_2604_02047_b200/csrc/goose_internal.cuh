@@ -30,6 +30,7 @@ struct goose_ctx {
     // top-k workspace
     unsigned long long* topk_cand;   // [topk_rows_cap][topk_chunks_cap][kMaxK]
     int32_t* row_counters;    // [topk_rows_cap]
+    float* topk_lse_ws;       // [topk_rows_cap][chunks][2]: per-chunk (max, sum) of the log-sum-exp
     int64_t topk_cand_cap;    // elements
     int topk_rows_cap;
     // per-sequence status words
@@ -68,7 +69,10 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 
 // launchers (each returns a cudaError_t from the launch)
 cudaError_t launch_node_topk(goose_ctx* c, const __nv_bfloat16* logits, int rows, int V, int64_t ldl, int k,
-                             int32_t* argmax, int32_t* ids, float* vals, cudaStream_t st);
+                             int32_t* argmax, int32_t* ids, float* vals, float* row_lse, cudaStream_t st);
+cudaError_t launch_harvest_scatter(goose_ctx* c, const int32_t* row_tok, int rows, int table_rows, int k,
+                                   const int32_t* ids, const float* vals, const float* row_lse,
+                                   int32_t* adj_ids, float* adj_scores, cudaStream_t st);
 cudaError_t launch_accept(goose_ctx* c, const int32_t* draft_tok, const int32_t* parent, const int32_t* argmax,
                           int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus, cudaStream_t st);
 cudaError_t launch_kv_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* row_off,

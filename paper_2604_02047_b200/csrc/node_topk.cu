@@ -64,11 +64,16 @@ __device__ __forceinline__ uint32_t bits_of_sortable16(uint32_t s) {
 __device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t w) { return *reinterpret_cast<__nv_bfloat162*>(&w); }
 __device__ __forceinline__ uint32_t as_u32(__nv_bfloat162 v) { return *reinterpret_cast<uint32_t*>(&v); }
 
-template <int KCAP>
+// LSE = true additionally returns the row's log-sum-exp (for the softmax scores of the harvest): the second
+// pass sums exp(x - chunk max) over every element, chunks are merged like split softmax partials.
+template <int KCAP, bool LSE>
 __global__ void __launch_bounds__(kTopkThreads, 2)
 node_topk_kernel(const __nv_bfloat16* __restrict__ logits, int V, int64_t ldl, int k, int chunks,
                  u64* __restrict__ ws_cand, int32_t* __restrict__ row_counters,
-                 int32_t* __restrict__ argmax, int32_t* __restrict__ ids, float* __restrict__ vals) {
+                 int32_t* __restrict__ argmax, int32_t* __restrict__ ids, float* __restrict__ vals,
+                 float* __restrict__ row_lse, float2* __restrict__ ws_lse) {
+    __shared__ float s_sum[32];
+    __shared__ uint32_t s_cmax;
     __shared__ uint32_t s_cand[32 * KCAP];               // per-warp winners (thread maxima, or exact keys)
     __shared__ uint32_t s_list[kTopkListCap];            // fast path: keys of all elements >= threshold
     __shared__ u64 s_merge[kTopkMaxChunks * KCAP];
@@ -121,6 +126,7 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, int V, int64_t ldl, i
         uint32_t w = 0;
         for (int r = 0; r < k; ++r) {
             w = __reduce_max_sync(0xFFFFFFFFu, cur);
+            if (LSE && r == 0 && lane == 0) s_cmax = w;   // the chunk's maximum
             const uint32_t owners = __ballot_sync(0xFFFFFFFFu, cur == w);
             if (lane == __ffs(owners) - 1) {
                 ++ptr;
@@ -133,6 +139,8 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, int V, int64_t ldl, i
 
     // ---- phase 4: every element >= T becomes a full key (value image << 16 | 0xFFFF - index in chunk)
     const uint32_t thr_s = s_thresh;
+    float esum = 0.f;
+    const float cmax = LSE ? __uint_as_float(bits_of_sortable16(s_cmax) << 16) : 0.f;
     {
         const uint32_t tb = bits_of_sortable16(thr_s);
         const __nv_bfloat162 t2 = as_bf162(tb | (tb << 16));
@@ -140,6 +148,13 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, int V, int64_t ldl, i
         for (int it = 0; it < 4; ++it) {
             const uint4 v4 = load8(rowp, base + it * (kTopkThreads * 8) + tid * 8, V);
             const uint32_t wds[4] = {v4.x, v4.y, v4.z, v4.w};
+            if (LSE) {                                   // elements past V were loaded as -inf: exp gives 0
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    esum += exp2f((__uint_as_float(wds[q] << 16) - cmax) * 1.4426950408889634f);
+                    esum += exp2f((__uint_as_float(wds[q] & 0xFFFF0000u) - cmax) * 1.4426950408889634f);
+                }
+            }
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const uint32_t ge = __hge2_mask(as_bf162(wds[q]), t2);
@@ -157,8 +172,19 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, int V, int64_t ldl, i
             }
         }
     }
+    if (LSE) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) esum += __shfl_xor_sync(0xFFFFFFFFu, esum, o);
+        if (lane == 0) s_sum[warp] = esum;
+    }
     __syncthreads();
     const int n_list = s_count;
+    float csum = 0.f;                                    // warp 0: the chunk's sum of exp(x - cmax)
+    if (LSE && warp == 0) {
+        csum = s_sum[lane];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) csum += __shfl_xor_sync(0xFFFFFFFFu, csum, o);
+    }
 
     uint32_t mine = 0;                                   // warp 0: lane r ends up with the r-th winner
     if (n_list <= kTopkListCap) {
@@ -232,6 +258,7 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, int V, int64_t ldl, i
         // cross-chunk merge on 64-bit keys (value image << 32 | ~global index)
         u64* dst = ws_cand + ((size_t)row * chunks + chunk) * kMaxK;
         if (lane < k) dst[lane] = mine ? (((u64)my_sv << 32) | (u64)(0xFFFFFFFFu - (uint32_t)my_id)) : 0ull;
+        if (LSE && lane == 0) ws_lse[(size_t)row * chunks + chunk] = make_float2(cmax, csum);
         __threadfence();
         __syncwarp();
         if (lane == 0) {
@@ -259,6 +286,18 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, int V, int64_t ldl, i
         if (lane == 0) row_counters[row] = 0;               // ready for the next launch
         my_id = (int32_t)(0xFFFFFFFFu - (uint32_t)(win & 0xFFFFFFFFull));
         my_sv = (uint32_t)(win >> 32);
+        if (LSE && lane == 0) {
+            float M = -INFINITY;
+            for (int c = 0; c < chunks; ++c) M = fmaxf(M, __ldcg(&ws_lse[(size_t)row * chunks + c]).x);
+            float sum = 0.f;
+            for (int c = 0; c < chunks; ++c) {
+                const float2 ms = __ldcg(&ws_lse[(size_t)row * chunks + c]);
+                sum += ms.y * expf(ms.x - M);
+            }
+            row_lse[row] = M + logf(sum);
+        }
+    } else if (LSE && lane == 0) {
+        row_lse[row] = cmax + logf(csum);
     }
     if (lane < k) {
         ids[(size_t)row * k + lane] = my_id;
@@ -268,7 +307,7 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, int V, int64_t ldl, i
 }
 
 cudaError_t launch_node_topk(goose_ctx* c, const __nv_bfloat16* logits, int rows, int V, int64_t ldl, int k,
-                             int32_t* argmax, int32_t* ids, float* vals, cudaStream_t st) {
+                             int32_t* argmax, int32_t* ids, float* vals, float* row_lse, cudaStream_t st) {
     if (rows == 0) return cudaSuccess;
     int chunks = (V + kTopkChunk - 1) / kTopkChunk;
     for (int r0 = 0; r0 < rows; r0 += 65535) {               // gridDim.y limit
@@ -277,8 +316,12 @@ cudaError_t launch_node_topk(goose_ctx* c, const __nv_bfloat16* logits, int rows
         const __nv_bfloat16* lp = logits + (size_t)r0 * ldl;
         u64* ws = c->topk_cand + (size_t)r0 * chunks * kMaxK;
         float* vp = vals ? vals + (size_t)r0 * k : nullptr;
-        cudaError_t e = launch_pdl(k <= 8 ? node_topk_kernel<8> : node_topk_kernel<16>, grid, dim3(kTopkThreads), 0, st,
-                                   lp, V, ldl, k, chunks, ws, c->row_counters + r0, argmax + r0, ids + (size_t)r0 * k, vp);
+        float* lsep = row_lse ? row_lse + r0 : nullptr;
+        float2* wl = reinterpret_cast<float2*>(c->topk_lse_ws) + (size_t)r0 * chunks;
+        auto kern = row_lse ? (k <= 8 ? node_topk_kernel<8, true> : node_topk_kernel<16, true>)
+                            : (k <= 8 ? node_topk_kernel<8, false> : node_topk_kernel<16, false>);
+        cudaError_t e = launch_pdl(kern, grid, dim3(kTopkThreads), 0, st, lp, V, ldl, k, chunks, ws, c->row_counters + r0,
+                                   argmax + r0, ids + (size_t)r0 * k, vp, lsep, wl);
         c->launches++;
         if (e != cudaSuccess) return e;
     }
@@ -334,8 +377,8 @@ extern "C" int goose_node_topk_static(const void* logits, int rows, int V, int64
     if (chunks > 1 && cudaMemsetAsync(counters, 0, sizeof(int32_t) * (size_t)rows, st) != cudaSuccess)
         return GOOSE_ECUDA;
     dim3 grid(chunks, rows);                                             // rows <= 2048 < 65535
-    cudaError_t e = launch_pdl(k <= 8 ? node_topk_kernel<8> : node_topk_kernel<16>, grid, dim3(kTopkThreads), 0, st,
-                               static_cast<const __nv_bfloat16*>(logits), V, ldl, k, chunks, scratch,
-                               counters, argmax, topk_ids, topk_vals);
+    cudaError_t e = launch_pdl(k <= 8 ? node_topk_kernel<8, false> : node_topk_kernel<16, false>, grid, dim3(kTopkThreads), 0,
+                               st, static_cast<const __nv_bfloat16*>(logits), V, ldl, k, chunks, scratch, counters, argmax,
+                               topk_ids, topk_vals, static_cast<float*>(nullptr), static_cast<float2*>(nullptr));
     return e == cudaSuccess ? GOOSE_OK : GOOSE_ECUDA;
 }

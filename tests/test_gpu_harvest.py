@@ -1,0 +1,71 @@
+"""GPU parity of goose_harvest (top-k + row log-sum-exp + scatter into the Tier-1 adjacency table) against
+the oracle: ids bit-exact, softmax scores within 1e-5 relative (fp32 sum of exp2 vs fp64), lse within 2e-5."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2604_02047_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def goose():
+    from paper_2604_02047_b200 import binding, build
+    build.build()
+    g = binding.Goose(max_S=16, max_B=128, max_H=8)
+    yield g
+    g.close()
+
+
+def _bf16(bits):
+    return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).cuda()
+
+
+def _check(goose, oracle, bits, k, tok, table_rows, V=None):
+    ids0 = np.full((table_rows, k), -7, np.int32); sc0 = np.full((table_rows, k), -1.0, np.float32)
+    adj_ids = torch.from_numpy(ids0).cuda(); adj_sc = torch.from_numpy(sc0).cuda()
+    am, ids, vals, lse = goose.harvest(_bf16(bits), k, torch.from_numpy(np.asarray(tok, np.int32)).cuda(), adj_ids, adj_sc, V=V)
+    torch.cuda.synchronize()
+    rids, rsc, rlse = oracle.harvest(bits, k, tok, ids0, sc0.astype(np.float64), V=V)
+    ram, rtop, rvals = oracle.node_topk(bits, k, V=V)
+    assert np.array_equal(am.cpu().numpy(), ram) and np.array_equal(ids.cpu().numpy(), rtop)
+    assert np.array_equal(vals.cpu().numpy().astype(np.float64), rvals)
+    assert np.abs(lse.cpu().numpy().astype(np.float64) - rlse).max() <= 2e-5
+    assert np.array_equal(adj_ids.cpu().numpy(), rids)                       # incl. untouched rows and last-writer rule
+    got = adj_sc.cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(got - rsc) <= 1e-5 * np.abs(rsc) + 1e-12)
+
+
+def test_harvest_tree_logits(goose, oracle):
+    for cid in (0, 1):
+        x = synth.make_config(cid)
+        _check(goose, oracle, x.logits, x.k, x.draft_tok.reshape(-1), x.V)
+
+
+def test_harvest_duplicates_and_bad_tokens(goose, oracle):
+    rng = np.random.default_rng(8)
+    rows, V, k = 300, 4096, 10
+    bits = synth.f32_to_bf16_bits((rng.standard_normal((rows, V)) * 2).astype(np.float32))
+    tok = rng.integers(0, 60, rows).astype(np.int32)                          # heavy duplication: 60 tokens, 300 rows
+    tok[5] = -1; tok[17] = V; tok[rows - 1] = tok[0]
+    _check(goose, oracle, bits, k, tok, V)
+
+
+def test_harvest_long_rows_and_row_stride(goose, oracle):
+    rng = np.random.default_rng(9)
+    rows, V, ldl, k = 9, 100001, 100008, 16                                   # four 32768-element chunks, ragged tail
+    bits = synth.f32_to_bf16_bits(rng.standard_normal((rows, ldl), dtype=np.float32))
+    bits[:, V:] = 0x7F00                                                     # padding must not enter the sums
+    _check(goose, oracle, bits, k, np.arange(rows, dtype=np.int32) * 11111, V, V=V)
+    const = np.full((2, 40000), 0x4040, np.uint16)                            # constant rows: slow path + lse = 3 + ln V
+    _check(goose, oracle, const, 8, [1, 2], 40000)
+
+
+def test_harvest_argument_errors(goose):
+    from paper_2604_02047_b200 import binding
+    lg = torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda")
+    tok = torch.zeros(4, dtype=torch.int32, device="cuda")
+    with pytest.raises(binding.GooseError):
+        goose.harvest(lg, 17, tok, torch.zeros((64, 17), dtype=torch.int32, device="cuda"),
+                      torch.zeros((64, 17), dtype=torch.float32, device="cuda"))

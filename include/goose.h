@@ -158,7 +158,8 @@ int goose_kv_compact(goose_ctx* ctx, void* k_cache, void* v_cache, int64_t kv_ro
                      int32_t* new_ctx_len, void* stream);
 
 /* The whole step on one stream, in data-flow order: tree attention, node top-k (rows = S*B),
- * acceptance walk, KV compaction.  Arguments as in the four calls above.                         */
+ * acceptance walk, KV compaction (the last two share one launch).  Arguments and results as in the
+ * four calls above.                                                                             */
 int goose_verify_step(goose_ctx* ctx, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
                       const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
                       const int32_t* draft_tok, const void* logits, int64_t ldl,

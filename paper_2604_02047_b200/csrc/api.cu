@@ -228,10 +228,12 @@ int goose_verify_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache,
     if (rc) return rc;
     rc = goose_node_topk(c, logits, S * B, V, ldl, k, argmax, topk_ids, topk_vals, stream);
     if (rc) return rc;
-    rc = goose_accept(c, draft_tok, parent, argmax, S, B, path, accept_len, bonus, stream);
-    if (rc) return rc;
-    return goose_kv_compact(c, k_cache, v_cache, kv_rows, row_off, ctx_len, path, accept_len, S, B, H, D,
-                            new_ctx_len, stream);
+    // acceptance walk + compaction in one launch (same results as goose_accept followed by goose_kv_compact)
+    cudaError_t e = goose::launch_accept_compact(c, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, row_off, ctx_len,
+                                                 draft_tok, parent, argmax, S, B, H, path, accept_len, bonus,
+                                                 new_ctx_len, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e);
+    return GOOSE_OK;
 }
 
 int goose_verify_step_host(goose_ctx* c, void* k_cache, void* v_cache, int64_t kv_rows,

@@ -76,4 +76,108 @@ cudaError_t launch_kv_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc
     return e;
 }
 
+// ---------------------------------------------------------------------------------------------------
+// Fused form used by goose_verify_step: the acceptance walk (Algorithm 3) and the compaction in one launch.
+// Every CTA redoes the walk of its sequence with warp 0 (a handful of warp reductions) instead of waiting for
+// a separate kernel; CTA (0, 0, s) publishes path / accept_len / bonus / new_ctx.
+__global__ void __launch_bounds__(kCompactThreads)
+accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __restrict__ row_off,
+                      const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ draft_tok,
+                      const int32_t* __restrict__ parent, const int32_t* __restrict__ argmax,
+                      int B, int row_vec, int32_t* __restrict__ path, int32_t* __restrict__ accept_len,
+                      int32_t* __restrict__ bonus, int32_t* __restrict__ new_ctx, int32_t* __restrict__ status) {
+    __shared__ int s_path[kMaxB];
+    __shared__ int s_len;
+    const int s = blockIdx.z;
+    const int which = blockIdx.y;                        // 0 = K, 1 = V
+    const int col = blockIdx.x * kCompactThreads + threadIdx.x;
+    const bool publisher = blockIdx.x == 0 && which == 0;
+    pdl_wait();
+    pdl_trigger();
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x;
+        const int32_t* par = parent + (size_t)s * B;
+        const int32_t* tok = draft_tok + (size_t)s * B;
+        const int32_t* am = argmax + (size_t)s * B;
+        constexpr int kPer = kMaxB / 32;
+        int my_par[kPer];
+        bool my_match[kPer];
+        bool bad = false;
+#pragma unroll
+        for (int t = 0; t < kPer; ++t) {
+            const int c = lane + 32 * t;
+            my_par[t] = -2;
+            my_match[t] = false;
+            if (c < B) {
+                const int pp = par[c];
+                my_par[t] = pp;
+                bad |= (c == 0) ? (pp != -1) : (pp < 0 || pp >= c);
+            }
+        }
+        bad = __any_sync(0xFFFFFFFFu, bad);
+        for (int c = lane; c < B; c += 32) s_path[c] = (c == 0) ? 0 : -1;
+        __syncwarp();
+        int v = 0, len = 0;
+        if (!bad) {
+#pragma unroll
+            for (int t = 0; t < kPer; ++t) {
+                const int c = lane + 32 * t;
+                if (c >= 1 && c < B) my_match[t] = (tok[c] == am[my_par[t]]);
+            }
+            for (int step = 0; step < B - 1; ++step) {
+                int cand = 0x7FFFFFFF;
+#pragma unroll
+                for (int t = kPer - 1; t >= 0; --t)
+                    if (my_match[t] && my_par[t] == v) cand = lane + 32 * t;
+                cand = __reduce_min_sync(0xFFFFFFFFu, cand);
+                if (cand == 0x7FFFFFFF) break;
+                ++len;
+                if (lane == 0) s_path[len] = cand;
+                v = cand;
+            }
+        }
+        __syncwarp();
+        if (lane == 0) s_len = len;
+        if (publisher) {
+            for (int c = lane; c < B; c += 32) path[(size_t)s * B + c] = s_path[c];
+            if (lane == 0) {
+                accept_len[s] = len;
+                bonus[s] = bad ? -1 : am[v];
+                new_ctx[s] = ctx_len[s] + 1 + len;
+                if (bad) atomicOr(&status[s], GOOSE_ST_BAD_PARENT);
+            }
+        }
+    }
+    __syncthreads();
+    const int L = s_len;
+    if (col >= row_vec) return;
+    uint4* base = reinterpret_cast<uint4*>(which ? vc : kc) + ((size_t)(row_off[s] + ctx_len[s])) * row_vec + col;
+    for (int j0 = 1; j0 <= L; j0 += kCompactBatch) {
+        uint4 r[kCompactBatch];
+#pragma unroll
+        for (int t = 0; t < kCompactBatch; ++t) {
+            const int j = j0 + t;
+            if (j <= L && s_path[j] != j) r[t] = base[(size_t)s_path[j] * row_vec];
+        }
+#pragma unroll
+        for (int t = 0; t < kCompactBatch; ++t) {
+            const int j = j0 + t;
+            if (j <= L && s_path[j] != j) base[(size_t)j * row_vec] = r[t];
+        }
+    }
+}
+
+cudaError_t launch_accept_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* row_off,
+                                  const int32_t* ctx_len, const int32_t* draft_tok, const int32_t* parent,
+                                  const int32_t* argmax, int S, int B, int H, int32_t* path, int32_t* accept_len,
+                                  int32_t* bonus, int32_t* new_ctx, cudaStream_t st) {
+    if (S == 0) return cudaSuccess;
+    int row_vec = H * kHeadDim * 2 / 16;
+    dim3 grid((row_vec + kCompactThreads - 1) / kCompactThreads, 2, S);
+    cudaError_t e = launch_pdl(accept_compact_kernel, grid, dim3(kCompactThreads), 0, st, kc, vc, row_off, ctx_len,
+                               draft_tok, parent, argmax, B, row_vec, path, accept_len, bonus, new_ctx, c->status);
+    c->launches++;
+    return e;
+}
+
 }  // namespace goose

@@ -187,6 +187,37 @@ int goose_verify_step_host(goose_ctx* ctx, void* k_cache, void* v_cache, int64_t
                            int32_t* h_path, int32_t* h_accept_len, int32_t* h_bonus,
                            int32_t* h_new_ctx_len, void* stream);
 
+/* ---- host routines of the loop around the verification step (all pointers below are HOST pointers) ---- */
+
+/* BuildSpineTree (Algorithm 1).  anchor = the last accepted token (spine root); chain[m] = the context-match
+ * draft; adj_ids int32 [table_rows][K] = Tier-1 adjacency table ids in rank order (negative = empty slot).
+ * Budget: b_s = min(m, floor(B r)), b_r = floor((B-1-b_s)(1-rho)), b_rho = B-1-b_s-b_r; step 1 lays the spine,
+ * step 2 attaches up to b_r ranked successors of the anchor to the root, step 3 attaches
+ * a_i = floor(b_rho (1/i) / H_{b_s}) successors of spine token d_i to spine node i, step 4 extends every branch leaf
+ * breadth-first by its top successor up to D nodes per branch while nodes remain.  Successors that would
+ * duplicate a sibling (e.g. the spine continuation) are skipped.  Output in spine-first topological order
+ * (parent[i] < i): draft_tok, parent (capacity B), is_spine (may be NULL), *n_nodes <= B, *n_spine = b_s + 1.  */
+int goose_build_spine_tree(int32_t anchor, const int32_t* chain, int m, const int32_t* adj_ids, int table_rows, int K,
+                           int B, int D, float r, float rho, int32_t* draft_tok, int32_t* parent, uint8_t* is_spine,
+                           int32_t* n_nodes, int32_t* n_spine);
+
+/* Fill nodes n_nodes..B-1 with padding (children of the root with negative tokens, which no argmax can match), so
+ * that a tree with fewer than B nodes can be verified by kernels that take a fixed B.                           */
+int goose_pad_tree(int32_t* draft_tok, int32_t* parent, int n_nodes, int B);
+
+/* ContextMatch (paragraph after Algorithm 2): n-gram lookup with n in {5, 4, 3} of the last n tokens of ctx at
+ * their most recent earlier occurrence; chain = the continuation (at most max_len tokens) of the longest n that
+ * matched, *chain_len = 0 if none; *consensus = 1 iff at least two n's matched and agree on the first
+ * continuation token.                                                                                           */
+int goose_context_match(const int32_t* ctx, int n_ctx, int max_len, int32_t* chain, int32_t* chain_len,
+                        int32_t* consensus);
+
+/* Spine-ratio tier (hyper-parameter table): p_hat < 0.2 -> 0.15, < 0.4 -> 0.30, otherwise 0.50.                  */
+float goose_spine_ratio_tier(float p_hat);
+
+/* EMA of the spine acceptance rate, coefficient 0.3: 0.7 p_hat + 0.3 accepted/drafted (unchanged if drafted = 0). */
+float goose_spine_ema(float p_hat, int accepted_spine, int drafted_spine);
+
 /* Synchronise the device, copy the per-sequence status words (GOOSE_ST_* bits, OR-ed over all
  * calls since the last query) into host_status[0..S) (a HOST array) and clear them.
  * Returns GOOSE_ETIMEOUT if any word has GOOSE_ST_TIMEOUT set.  For tests and debugging.         */

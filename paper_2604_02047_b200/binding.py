@@ -20,6 +20,7 @@ EXPORTS = [
     "goose_create", "goose_destroy", "goose_strerror", "goose_set_attn_impl", "goose_tree_attn",
     "goose_node_topk", "goose_accept", "goose_kv_compact", "goose_verify_step",
     "goose_verify_step_host", "goose_last_status", "goose_launch_count", "goose_node_topk_static", "goose_harvest",
+    "goose_build_spine_tree", "goose_pad_tree", "goose_context_match", "goose_spine_ratio_tier", "goose_spine_ema",
 ]
 
 ATTN_AUTO, ATTN_MMA, ATTN_UMMA = 0, 1, 2
@@ -46,8 +47,12 @@ def load_library() -> ctypes.CDLL:
     lib.goose_launch_count.restype = ctypes.c_int64
     lib.goose_launch_count.argtypes = [ctypes.c_void_p]
     for name in EXPORTS:
-        if name not in ("goose_strerror", "goose_launch_count"):
+        if name not in ("goose_strerror", "goose_launch_count", "goose_spine_ratio_tier", "goose_spine_ema"):
             getattr(lib, name).restype = ctypes.c_int
+    lib.goose_spine_ratio_tier.restype = ctypes.c_float
+    lib.goose_spine_ratio_tier.argtypes = [ctypes.c_float]
+    lib.goose_spine_ema.restype = ctypes.c_float
+    lib.goose_spine_ema.argtypes = [ctypes.c_float, ctypes.c_int, ctypes.c_int]
     _lib = lib
     return lib
 
@@ -244,6 +249,40 @@ def node_topk_static(logits: torch.Tensor, k: int, V: Optional[int] = None, want
                                           ctypes.c_int(k), _p(argmax), _p(ids), _p(vals), _stream()),
                "goose_node_topk_static")
     return argmax, ids, vals
+
+
+# ---------------------------------------------------------------------- host routines (numpy in, numpy out)
+def build_spine_tree(anchor: int, chain, adj_ids, B: int, D: int, r: float, rho: float, pad: bool = False):
+    """``goose_build_spine_tree`` (+ ``goose_pad_tree``).  adj_ids: int32 numpy [table_rows][K] on the host.
+    Returns (draft_tok, parent, is_spine, n_nodes, n_spine); arrays have length B when ``pad`` else n_nodes."""
+    import numpy as np
+    lib = load_library()
+    chain = np.ascontiguousarray(chain, dtype=np.int32)
+    adj_ids = np.ascontiguousarray(adj_ids, dtype=np.int32)
+    tok = np.zeros(B, np.int32); par = np.zeros(B, np.int32); sp = np.zeros(B, np.uint8)
+    n = ctypes.c_int32(); ns = ctypes.c_int32()
+    vp = lambda a: a.ctypes.data_as(ctypes.c_void_p)
+    _check(lib.goose_build_spine_tree(ctypes.c_int32(anchor), vp(chain), ctypes.c_int(len(chain)), vp(adj_ids),
+                                      ctypes.c_int(adj_ids.shape[0]), ctypes.c_int(adj_ids.shape[1]), ctypes.c_int(B),
+                                      ctypes.c_int(D), ctypes.c_float(r), ctypes.c_float(rho), vp(tok), vp(par), vp(sp),
+                                      ctypes.byref(n), ctypes.byref(ns)), "goose_build_spine_tree")
+    if pad:
+        _check(lib.goose_pad_tree(vp(tok), vp(par), n, ctypes.c_int(B)), "goose_pad_tree")
+        return tok, par, sp.astype(bool), n.value, ns.value
+    return tok[:n.value], par[:n.value], sp[:n.value].astype(bool), n.value, ns.value
+
+
+def context_match(ctx, max_len: int = 20):
+    """``goose_context_match``: returns (chain, consensus)."""
+    import numpy as np
+    lib = load_library()
+    ctx = np.ascontiguousarray(ctx, dtype=np.int32)
+    chain = np.zeros(max(1, max_len), np.int32)
+    n = ctypes.c_int32(); c = ctypes.c_int32()
+    vp = lambda a: a.ctypes.data_as(ctypes.c_void_p)
+    _check(lib.goose_context_match(vp(ctx), ctypes.c_int(len(ctx)), ctypes.c_int(max_len), vp(chain), ctypes.byref(n),
+                                   ctypes.byref(c)), "goose_context_match")
+    return chain[:n.value].tolist(), bool(c.value)
 
 
 # ---------------------------------------------------------------------- helpers for tests / bench

@@ -167,7 +167,8 @@ def run_reference(args, x, cfg_name):
     """--impl reference: the oracle (the only reference there is), on the host cores, rank 0 only."""
     res = None
     for i in range(args.warmup + args.steps):
-        r = oracle_sample(x, budget_s=max(1.0, min(12.0, 90.0 / max(1, args.warmup + args.steps))))
+        # bounded sample per step so that warm-up + K steps stay within a few minutes of host time
+        r = oracle_sample(x, budget_s=max(0.15, min(12.0, 100.0 / max(1, args.warmup + args.steps))))
         if i >= args.warmup:
             res = r if res is None else {**r, "step_s": res["step_s"] + r["step_s"]}
     step_s = res["step_s"] / args.steps
@@ -233,7 +234,7 @@ def run_ours(args, x, cfg, rank, world, local_rank):
         def capture(fn):
             gr = torch.cuda.CUDAGraph()
             n0 = g.launch_count()
-            with torch.cuda.graph(gr, stream=stream):
+            with torch.cuda.graph(gr, stream=stream, capture_error_mode="thread_local"):
                 for i in range(R):
                     fn(i)
             return gr, (g.launch_count() - n0) // R

@@ -223,6 +223,13 @@ float goose_spine_ema(float p_hat, int accepted_spine, int drafted_spine);
  * Returns GOOSE_ETIMEOUT if any word has GOOSE_ST_TIMEOUT set.  For tests and debugging.         */
 int goose_last_status(goose_ctx* ctx, int32_t* host_status, int S);
 
+/* Self-test of the device-side time-out path.  Runs a one-warp kernel whose wait (the same bounded mbarrier wait
+ * the attention kernel uses) can never be satisfied and gives up after `limit_cycles` SM cycles (keep it short, e.g.
+ * 1e6 = about half a millisecond).  Returns GOOSE_OK when the wait reported failure and the kernel returned
+ * normally; afterwards goose_last_status shows GOOSE_ST_TIMEOUT in word 0 (and returns GOOSE_ETIMEOUT), and the
+ * context remains fully usable.  Synchronises `stream`.                                                         */
+int goose_selftest_bounded_wait(goose_ctx* ctx, int64_t limit_cycles, void* stream);
+
 /* Number of kernels this library has launched through `ctx` since it was created.              */
 int64_t goose_launch_count(goose_ctx* ctx);
 

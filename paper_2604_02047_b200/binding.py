@@ -21,6 +21,7 @@ EXPORTS = [
     "goose_node_topk", "goose_accept", "goose_kv_compact", "goose_verify_step",
     "goose_verify_step_host", "goose_last_status", "goose_launch_count", "goose_node_topk_static", "goose_harvest",
     "goose_build_spine_tree", "goose_pad_tree", "goose_context_match", "goose_spine_ratio_tier", "goose_spine_ema",
+    "goose_selftest_bounded_wait",
 ]
 
 ATTN_AUTO, ATTN_MMA, ATTN_UMMA = 0, 1, 2
@@ -111,6 +112,10 @@ class Goose:
 
     def launch_count(self) -> int:
         return int(self.lib.goose_launch_count(self.h))
+
+    def selftest_bounded_wait(self, limit_cycles: int = 1_000_000) -> int:
+        """Run the time-out self-test; returns the library's return code (0 = the wait gave up as designed)."""
+        return int(self.lib.goose_selftest_bounded_wait(self.h, ctypes.c_int64(limit_cycles), _stream()))
 
     def last_status(self, S: int) -> torch.Tensor:
         st = torch.zeros(S, dtype=torch.int32)

@@ -315,6 +315,20 @@ int goose_verify_step_host(goose_ctx* c, void* k_cache, void* v_cache, int64_t k
     return GOOSE_OK;
 }
 
+int goose_selftest_bounded_wait(goose_ctx* c, int64_t limit_cycles, void* stream) {
+    if (!c || limit_cycles < 1 || limit_cycles > 4000000000LL) return GOOSE_EINVAL;
+    GOOSE_CUDA(cudaSetDevice(c->device));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t* d_result = reinterpret_cast<int32_t*>(c->row_counters);   // idle scratch word between top-k launches
+    GOOSE_CUDA(cudaStreamSynchronize(st));
+    GOOSE_CUDA(goose::launch_bounded_wait_selftest(c, limit_cycles, d_result, st));
+    int32_t h_result = -1;
+    GOOSE_CUDA(cudaMemcpyAsync(&h_result, d_result, sizeof h_result, cudaMemcpyDeviceToHost, st));
+    GOOSE_CUDA(cudaMemsetAsync(d_result, 0, sizeof(int32_t), st));       // the counter must be zero for top-k
+    GOOSE_CUDA(cudaStreamSynchronize(st));
+    return h_result == 0 ? GOOSE_OK : GOOSE_ECUDA;
+}
+
 int goose_last_status(goose_ctx* c, int32_t* host_status, int S) {
     if (!c || !host_status || S < 0 || S > c->max_S) return GOOSE_EINVAL;
     GOOSE_CUDA(cudaSetDevice(c->device));

@@ -13,7 +13,8 @@ constexpr int kHeadDim = GOOSE_HEAD_DIM;
 constexpr int kMaxB = GOOSE_MAX_B;
 constexpr int kMaxK = GOOSE_MAX_K;
 
-// Workspace layout of one split-KV partial: O fp32 [kMaxB][128] (unnormalised), then m[kMaxB], l[kMaxB].
+// Workspace slot of one split-KV partial.  The mma kernel stores O fp32 [kMaxB][128] (unnormalised), then m[kMaxB],
+// l[kMaxB]; the tcgen05 kernel uses the first half of a slot for its fp16 layout (see tree_attn_umma.cu).
 constexpr int kPartialFloats = kMaxB * kHeadDim + 2 * kMaxB;
 
 }  // namespace goose
@@ -91,8 +92,9 @@ cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __
                                   const int32_t* ctx_len, const int32_t* parent, int S, int B, int H,
                                   float scale, __nv_bfloat16* out, float* lse, cudaStream_t st);
 
-// Max context rows assumed when sizing the fixed-split grid of the mma kernel is not needed:
-// ctx_len lives on the device, so the split count depends only on S, H and the SM count.
+cudaError_t launch_bounded_wait_selftest(goose_ctx* c, long long limit_cycles, int32_t* result, cudaStream_t st);
+
+// split count of the mma kernel's fixed grid: ctx_len lives on the device, so it depends only on S, H and the SM count
 int mma_splits(const goose_ctx* c, int S, int H);
 
 // per-device kernel attributes (dynamic shared memory limits); called once from goose_create

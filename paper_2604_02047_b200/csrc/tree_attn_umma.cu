@@ -102,19 +102,24 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t 
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait (about one second of SM clock).  Returns false, and raises the CTA's abort flag, when it
-// gives up; returns false at once when another role has already aborted.
-__device__ __forceinline__ bool mbar_wait(Header* hd, unsigned long long* bar, uint32_t parity, int32_t* status) {
+// Bounded wait.  Returns false, and raises the CTA's abort flag, when `limit` SM cycles pass without the barrier
+// completing; returns false at once when another role has already aborted.
+__device__ __forceinline__ bool mbar_wait_limit(Header* hd, unsigned long long* bar, uint32_t parity, int32_t* status,
+                                                long long limit) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
         if (hd->abort_flag) return false;
         if (mbar_try_wait(bar, parity)) return true;
-        if (clock64() - t0 > kWaitCycles) break;
+        if (clock64() - t0 > limit) break;
     }
     hd->abort_flag = 1;
     atomicOr(status, GOOSE_ST_TIMEOUT);
     return false;
+}
+// every wait of the attention kernel: about one second of SM clock
+__device__ __forceinline__ bool mbar_wait(Header* hd, unsigned long long* bar, uint32_t parity, int32_t* status) {
+    return mbar_wait_limit(hd, bar, parity, status, kWaitCycles);
 }
 // Bounded wait used only while draining after an abort (ignores the abort flag).
 __device__ __forceinline__ void mbar_drain(unsigned long long* bar, uint32_t parity) {
@@ -777,6 +782,32 @@ extern "C" int goose_debug_set_trace(void* dev_ptr) {
     return (int)cudaMemcpyToSymbol(g_trace, &p, sizeof p);
 }
 #endif
+
+// Self-test of the bounded-wait path: one warp waits on a barrier that nothing ever completes, with a short
+// limit.  The wait must give up, set GOOSE_ST_TIMEOUT in status[0] and let the kernel return normally, the same way
+// a stalled pipeline of the attention kernel would.  Nothing here can hang: the only loop is the bounded wait.
+__global__ void __launch_bounds__(32)
+bounded_wait_selftest_kernel(int32_t* __restrict__ status, long long limit_cycles, int32_t* __restrict__ result) {
+    __shared__ Header hd;
+    if (threadIdx.x == 0) {
+        mbar_init(&hd.pv_done, 1);
+        hd.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    bool ok = true;
+    if (threadIdx.x == 0) ok = mbar_wait_limit(&hd, &hd.pv_done, 0, status, limit_cycles);   // never completes
+    __syncwarp();
+    // the other lanes see the abort flag at once, as the other roles of the attention kernel would
+    if (threadIdx.x != 0) ok = mbar_wait_limit(&hd, &hd.pv_done, 0, status, limit_cycles);
+    if (threadIdx.x == 1) result[0] = ok ? 1 : 0;         // 0 expected: the wait reported failure, the kernel returns
+}
+
+cudaError_t launch_bounded_wait_selftest(goose_ctx* c, long long limit_cycles, int32_t* result, cudaStream_t st) {
+    bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(c->status, limit_cycles, result);
+    c->launches++;
+    return cudaGetLastError();
+}
 
 cudaError_t init_umma_kernel() {
     return cudaFuncSetAttribute(tree_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmem);

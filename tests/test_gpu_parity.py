@@ -317,6 +317,19 @@ def test_verify_step_host_buffers(goose, oracle):
                                                  V=1024, seed=3), host=True)
 
 
+def test_a_wait_that_cannot_be_satisfied_times_out_and_the_context_stays_usable(goose, oracle):
+    """Failure detection without a fault: the bounded wait gives up, reports GOOSE_ST_TIMEOUT, the kernel returns."""
+    from paper_2604_02047_b200 import binding
+    assert goose.selftest_bounded_wait(1_000_000) == 0                  # ~0.5 ms limit
+    st = torch.zeros(1, dtype=torch.int32)
+    rc = goose.lib.goose_last_status(goose.h, binding._p(st), 1)
+    assert rc == -4 and int(st[0]) & binding.ST_TIMEOUT                 # GOOSE_ETIMEOUT, status word set
+    assert not goose.last_status(1).any()                               # cleared by the query
+    x = synth.make_inputs(1, 2, 16, [140], [synth.kary_tree(16, 3)], V=64, seed=5)
+    _check_attn_full(goose, oracle, x, binding.ATTN_UMMA)               # the same context still works
+    _check_topk(goose, oracle, x.logits, 4)
+
+
 def test_host_side_argument_errors(goose):
     from paper_2604_02047_b200 import binding
     x = synth.make_config(0)

@@ -519,9 +519,15 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                             for (int c = 0; c < 128; ++c)
                                 v[c] = ((vw[c >> 5] >> (c & 31)) & 1u) ? v[c] : 0xFF800000u;   // -inf
                         }
-                        float mx = -INFINITY;
+                        // one warp per scheduler: nothing hides a serial chain, so the row maximum (and the row
+                        // sum below) run as four independent chains
+                        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                        for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(v[c]));
+                        for (int c = 0; c < 128; c += 4) {
+                            mx4[0] = fmaxf(mx4[0], __uint_as_float(v[c]));     mx4[1] = fmaxf(mx4[1], __uint_as_float(v[c + 1]));
+                            mx4[2] = fmaxf(mx4[2], __uint_as_float(v[c + 2])); mx4[3] = fmaxf(mx4[3], __uint_as_float(v[c + 3]));
+                        }
+                        float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                         mx *= scale_log2;                  // scale > 0
                         const float m_new = fmaxf(m_run, mx);
                         // lazy rescaling: keep the stale maximum unless it grew by more than the threshold
@@ -555,7 +561,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                     if (ok && jg > 0) ok = mbar_wait(hd, &hd->pv_done, (jg - 1) & 1, status);
                     if (!ok) break;
                     if (warp_has_rows) {
-                        float lsum = 0.f;
+                        float ls4[4] = {0.f, 0.f, 0.f, 0.f};
                         const float neg_m = -m_use;
                         unsigned char* prow = p_smem + row * 128;
 #pragma unroll
@@ -565,14 +571,14 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                             for (int e = 0; e < 4; ++e) {
                                 float p0 = ex2(fmaf(__uint_as_float(v[ch * 8 + 2 * e]), scale_log2, neg_m));
                                 float p1 = ex2(fmaf(__uint_as_float(v[ch * 8 + 2 * e + 1]), scale_log2, neg_m));
-                                lsum += p0 + p1;
+                                ls4[e] += p0 + p1;
                                 pk[e] = pack_bf16x2(p0, p1);
                             }
                             const int half = ch >> 3, cin = ch & 7;
                             *reinterpret_cast<uint4*>(prow + half * kHalfBytes + ((cin ^ (row & 7)) << 4)) =
                                 make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         }
-                        l_run += lsum;
+                        l_run += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
                     }
                     // ragged end: V rows past the sequence's last key may hold anything -> zero them
                     if ((t + 1) * kTile > n_keys) {

@@ -55,6 +55,7 @@ extern "C" {
 #define GOOSE_ST_BAD_PARENT   1   /* parent[] is not a rooted tree in topological order */
 #define GOOSE_ST_BAD_PATH     2   /* path[] / accept_len[] handed to goose_kv_compact is invalid */
 #define GOOSE_ST_TIMEOUT      4   /* a device-side wait ran out of polls */
+#define GOOSE_ST_BAD_ROWS     8   /* row_off[] / ctx_len[] put a sequence's rows outside [0, kv_rows): nothing moved */
 
 /* attention kernel selection (goose_set_attn_impl) */
 #define GOOSE_ATTN_AUTO  0

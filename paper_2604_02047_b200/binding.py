@@ -25,7 +25,7 @@ EXPORTS = [
 ]
 
 ATTN_AUTO, ATTN_MMA, ATTN_UMMA = 0, 1, 2
-ST_BAD_PARENT, ST_BAD_PATH, ST_TIMEOUT = 1, 2, 4
+ST_BAD_PARENT, ST_BAD_PATH, ST_TIMEOUT, ST_BAD_ROWS = 1, 2, 4, 8
 
 _lib: Optional[ctypes.CDLL] = None
 

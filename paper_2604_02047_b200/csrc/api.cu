@@ -87,6 +87,7 @@ int goose_create(goose_ctx** out, int device, int max_S, int max_B, int max_H, i
     ok = ok && cudaMalloc(&c->row_counters, sizeof(int32_t) * (size_t)c->topk_rows_cap) == cudaSuccess;
     ok = ok && cudaMalloc(&c->topk_lse_ws, sizeof(float) * 2 * (size_t)c->topk_rows_cap * kTopkMaxChunks) == cudaSuccess;
     ok = ok && cudaMalloc(&c->status, sizeof(int32_t) * (size_t)max_S) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->selftest_word, sizeof(int32_t)) == cudaSuccess;
     if (ok) {
         ok = ok && cudaMemset(c->head_counters, 0, sizeof(int32_t) * (size_t)heads) == cudaSuccess;
         ok = ok && cudaMemset(c->row_counters, 0, sizeof(int32_t) * (size_t)c->topk_rows_cap) == cudaSuccess;
@@ -113,7 +114,7 @@ int goose_destroy(goose_ctx* c) {
     if (!c) return GOOSE_EINVAL;
     cudaSetDevice(c->device);
     cudaFree(c->partials); cudaFree(c->head_counters); cudaFree(c->topk_cand);
-    cudaFree(c->row_counters); cudaFree(c->topk_lse_ws); cudaFree(c->status); cudaFree(c->stage);
+    cudaFree(c->row_counters); cudaFree(c->topk_lse_ws); cudaFree(c->status); cudaFree(c->selftest_word); cudaFree(c->stage);
     delete c;
     return GOOSE_OK;
 }
@@ -146,7 +147,7 @@ int goose_tree_attn(goose_ctx* c, const void* q, const void* k_cache, const void
                                          scale, (__nv_bfloat16*)out, lse, st);
     else
         e = goose::launch_tree_attn_mma(c, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_cache,
-                                        (const __nv_bfloat16*)v_cache, row_off, ctx_len, parent, S, B, H, scale,
+                                        (const __nv_bfloat16*)v_cache, kv_rows, row_off, ctx_len, parent, S, B, H, scale,
                                         (__nv_bfloat16*)out, lse, st);
     if (e != cudaSuccess) return cuda_fail(e);
     return GOOSE_OK;
@@ -201,7 +202,7 @@ int goose_kv_compact(goose_ctx* c, void* k_cache, void* v_cache, int64_t kv_rows
     if (!k_cache || !v_cache || !row_off || !ctx_len || !path || !accept_len || !new_ctx_len) return GOOSE_EINVAL;
     if (!aligned16(k_cache) || !aligned16(v_cache) || kv_rows < 1) return GOOSE_EINVAL;
     cudaError_t e = goose::launch_kv_compact(c, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, row_off, ctx_len,
-                                             path, accept_len, S, B, H, new_ctx_len,
+                                             path, accept_len, S, B, H, kv_rows, new_ctx_len,
                                              static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(e);
     return GOOSE_OK;
@@ -230,7 +231,7 @@ int goose_verify_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache,
     if (rc) return rc;
     // acceptance walk + compaction in one launch (same results as goose_accept followed by goose_kv_compact)
     cudaError_t e = goose::launch_accept_compact(c, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, row_off, ctx_len,
-                                                 draft_tok, parent, argmax, S, B, H, path, accept_len, bonus,
+                                                 draft_tok, parent, argmax, S, B, H, kv_rows, path, accept_len, bonus,
                                                  new_ctx_len, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(e);
     return GOOSE_OK;
@@ -319,12 +320,10 @@ int goose_selftest_bounded_wait(goose_ctx* c, int64_t limit_cycles, void* stream
     if (!c || limit_cycles < 1 || limit_cycles > 4000000000LL) return GOOSE_EINVAL;
     GOOSE_CUDA(cudaSetDevice(c->device));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    int32_t* d_result = reinterpret_cast<int32_t*>(c->row_counters);   // idle scratch word between top-k launches
-    GOOSE_CUDA(cudaStreamSynchronize(st));
+    int32_t* d_result = c->selftest_word;
     GOOSE_CUDA(goose::launch_bounded_wait_selftest(c, limit_cycles, d_result, st));
     int32_t h_result = -1;
     GOOSE_CUDA(cudaMemcpyAsync(&h_result, d_result, sizeof h_result, cudaMemcpyDeviceToHost, st));
-    GOOSE_CUDA(cudaMemsetAsync(d_result, 0, sizeof(int32_t), st));       // the counter must be zero for top-k
     GOOSE_CUDA(cudaStreamSynchronize(st));
     return h_result == 0 ? GOOSE_OK : GOOSE_ECUDA;
 }

@@ -36,6 +36,7 @@ struct goose_ctx {
     int topk_rows_cap;
     // per-sequence status words
     int32_t* status;          // [max_S]
+    int32_t* selftest_word;   // result word of goose_selftest_bounded_wait
     // host staging for goose_verify_step_host
     void* stage;              // device buffer
     size_t stage_bytes;
@@ -78,13 +79,13 @@ cudaError_t launch_accept(goose_ctx* c, const int32_t* draft_tok, const int32_t*
                           int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus, cudaStream_t st);
 cudaError_t launch_kv_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* row_off,
                               const int32_t* ctx_len, const int32_t* path, const int32_t* accept_len,
-                              int S, int B, int H, int32_t* new_ctx, cudaStream_t st);
+                              int S, int B, int H, int64_t kv_rows, int32_t* new_ctx, cudaStream_t st);
 cudaError_t launch_accept_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* row_off,
                                   const int32_t* ctx_len, const int32_t* draft_tok, const int32_t* parent,
-                                  const int32_t* argmax, int S, int B, int H, int32_t* path, int32_t* accept_len,
-                                  int32_t* bonus, int32_t* new_ctx, cudaStream_t st);
+                                  const int32_t* argmax, int S, int B, int H, int64_t kv_rows, int32_t* path,
+                                  int32_t* accept_len, int32_t* bonus, int32_t* new_ctx, cudaStream_t st);
 cudaError_t launch_tree_attn_mma(goose_ctx* c, const __nv_bfloat16* q, const __nv_bfloat16* kc,
-                                 const __nv_bfloat16* vc, const int64_t* row_off, const int32_t* ctx_len,
+                                 const __nv_bfloat16* vc, int64_t kv_rows, const int64_t* row_off, const int32_t* ctx_len,
                                  const int32_t* parent, int S, int B, int H, float scale,
                                  __nv_bfloat16* out, float* lse, cudaStream_t st);
 cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __nv_bfloat16* kc,

@@ -17,7 +17,7 @@ __global__ void __launch_bounds__(kCompactThreads)
 kv_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc,
                   const int64_t* __restrict__ row_off, const int32_t* __restrict__ ctx_len,
                   const int32_t* __restrict__ path, const int32_t* __restrict__ accept_len,
-                  int B, int row_vec /* 16-byte vectors per row = H*128*2/16 */,
+                  int B, int row_vec /* 16-byte vectors per row = H*128*2/16 */, int64_t kv_rows,
                   int32_t* __restrict__ new_ctx, int32_t* __restrict__ status) {
     __shared__ int s_path[kMaxB];
     __shared__ int s_bad;
@@ -30,7 +30,10 @@ kv_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc,
     int L = accept_len[s];
     if (threadIdx.x == 0) s_bad = 0;
     __syncthreads();
-    bool bad = (L < 0 || L >= B);
+    // rows this sequence owns must lie inside the cache: never form an address from unchecked device data
+    const int64_t r0 = row_off[s];
+    const bool bad_rows = ctx < 0 || r0 < 0 || r0 + ctx + B > kv_rows;
+    bool bad = (L < 0 || L >= B) || bad_rows;
     if (!bad) {
         for (int j = threadIdx.x; j <= L; j += kCompactThreads) {
             int pj = path[(size_t)s * B + j];
@@ -44,7 +47,7 @@ kv_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc,
     if (bad) L = 0;
     if (blockIdx.x == 0 && which == 0 && threadIdx.x == 0) {
         new_ctx[s] = ctx + 1 + L;
-        if (bad) atomicOr(&status[s], GOOSE_ST_BAD_PATH);
+        if (bad) atomicOr(&status[s], bad_rows ? GOOSE_ST_BAD_ROWS : GOOSE_ST_BAD_PATH);
     }
     if (bad || col >= row_vec) return;
 
@@ -66,12 +69,12 @@ kv_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc,
 
 cudaError_t launch_kv_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* row_off,
                               const int32_t* ctx_len, const int32_t* path, const int32_t* accept_len,
-                              int S, int B, int H, int32_t* new_ctx, cudaStream_t st) {
+                              int S, int B, int H, int64_t kv_rows, int32_t* new_ctx, cudaStream_t st) {
     if (S == 0) return cudaSuccess;
     int row_vec = H * kHeadDim * 2 / 16;
     dim3 grid((row_vec + kCompactThreads - 1) / kCompactThreads, 2, S);
     cudaError_t e = launch_pdl(kv_compact_kernel, grid, dim3(kCompactThreads), 0, st, kc, vc, row_off, ctx_len, path,
-                               accept_len, B, row_vec, new_ctx, c->status);
+                               accept_len, B, row_vec, kv_rows, new_ctx, c->status);
     c->launches++;
     return e;
 }
@@ -84,8 +87,9 @@ __global__ void __launch_bounds__(kCompactThreads)
 accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __restrict__ row_off,
                       const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ draft_tok,
                       const int32_t* __restrict__ parent, const int32_t* __restrict__ argmax,
-                      int B, int row_vec, int32_t* __restrict__ path, int32_t* __restrict__ accept_len,
-                      int32_t* __restrict__ bonus, int32_t* __restrict__ new_ctx, int32_t* __restrict__ status) {
+                      int B, int row_vec, int64_t kv_rows, int32_t* __restrict__ path,
+                      int32_t* __restrict__ accept_len, int32_t* __restrict__ bonus, int32_t* __restrict__ new_ctx,
+                      int32_t* __restrict__ status) {
     __shared__ int s_path[kMaxB];
     __shared__ int s_len;
     const int s = blockIdx.z;
@@ -94,6 +98,10 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
     const bool publisher = blockIdx.x == 0 && which == 0;
     pdl_wait();
     pdl_trigger();
+    // rows this sequence owns must lie inside the cache: never form an address from unchecked device data
+    const int ctx0 = ctx_len[s];
+    const int64_t r0 = row_off[s];
+    const bool bad_rows = ctx0 < 0 || r0 < 0 || r0 + ctx0 + B > kv_rows;
     if (threadIdx.x < 32) {
         const int lane = threadIdx.x;
         const int32_t* par = parent + (size_t)s * B;
@@ -143,15 +151,16 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
             if (lane == 0) {
                 accept_len[s] = len;
                 bonus[s] = bad ? -1 : am[v];
-                new_ctx[s] = ctx_len[s] + 1 + len;
+                new_ctx[s] = ctx0 + 1 + len;
                 if (bad) atomicOr(&status[s], GOOSE_ST_BAD_PARENT);
+                if (bad_rows) atomicOr(&status[s], GOOSE_ST_BAD_ROWS);
             }
         }
     }
     __syncthreads();
     const int L = s_len;
-    if (col >= row_vec) return;
-    uint4* base = reinterpret_cast<uint4*>(which ? vc : kc) + ((size_t)(row_off[s] + ctx_len[s])) * row_vec + col;
+    if (col >= row_vec || bad_rows) return;
+    uint4* base = reinterpret_cast<uint4*>(which ? vc : kc) + ((size_t)(r0 + ctx0)) * row_vec + col;
     for (int j0 = 1; j0 <= L; j0 += kCompactBatch) {
         uint4 r[kCompactBatch];
 #pragma unroll
@@ -169,13 +178,13 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
 
 cudaError_t launch_accept_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* row_off,
                                   const int32_t* ctx_len, const int32_t* draft_tok, const int32_t* parent,
-                                  const int32_t* argmax, int S, int B, int H, int32_t* path, int32_t* accept_len,
-                                  int32_t* bonus, int32_t* new_ctx, cudaStream_t st) {
+                                  const int32_t* argmax, int S, int B, int H, int64_t kv_rows, int32_t* path,
+                                  int32_t* accept_len, int32_t* bonus, int32_t* new_ctx, cudaStream_t st) {
     if (S == 0) return cudaSuccess;
     int row_vec = H * kHeadDim * 2 / 16;
     dim3 grid((row_vec + kCompactThreads - 1) / kCompactThreads, 2, S);
     cudaError_t e = launch_pdl(accept_compact_kernel, grid, dim3(kCompactThreads), 0, st, kc, vc, row_off, ctx_len,
-                               draft_tok, parent, argmax, B, row_vec, path, accept_len, bonus, new_ctx, c->status);
+                               draft_tok, parent, argmax, B, row_vec, kv_rows, path, accept_len, bonus, new_ctx, c->status);
     c->launches++;
     return e;
 }

@@ -87,7 +87,7 @@ __global__ void __launch_bounds__(256)
 tree_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ kc,
                      const __nv_bfloat16* __restrict__ vc, const int64_t* __restrict__ row_off,
                      const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ parent,
-                     int B, int H, float scale_log2, int splits,
+                     int B, int H, int64_t kv_rows, float scale_log2, int splits,
                      float* __restrict__ partials, int32_t* __restrict__ head_counters,
                      int32_t* __restrict__ status, __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -98,7 +98,7 @@ tree_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     const int g = lane >> 2, t4 = lane & 3;
     pdl_wait();
     pdl_trigger();
-    const int ctx = ctx_len[s];
+    const int ctx = max(ctx_len[s], 0);                    // device data: a negative length is treated as 0
     const int64_t row0 = row_off[s];
     const int n_keys = ctx + B;
     const int n_tiles = (n_keys + kKT - 1) / kKT;
@@ -112,7 +112,9 @@ tree_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
         int p = par[i];
         bad |= (i == 0) ? (p != -1) : (p < 0 || p >= i);
     }
-    bad = __syncthreads_or(bad);
+    // the sequence's rows must lie inside the cache: never form an address from unchecked device data
+    const bool bad_rows = ctx_len[s] < 0 || row0 < 0 || row0 + ctx + B > kv_rows;
+    bad = __syncthreads_or(bad | (bad_rows ? 1 : 0));
 
     const int rowA = warp * 16 + g, rowB = rowA + 8;       // this thread's two query rows
     const bool warp_active = (warp * 16 < B) && !bad;
@@ -231,7 +233,7 @@ tree_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
 
     if (splits == 1 || bad) {
         if (bad) {
-            if (tid == 0 && split == 0 && h == 0) atomicOr(&status[s], GOOSE_ST_BAD_PARENT);
+            if (tid == 0 && split == 0 && h == 0) atomicOr(&status[s], bad_rows ? GOOSE_ST_BAD_ROWS : GOOSE_ST_BAD_PARENT);
             // zero-fill this CTA's share of the head's output
             for (int idx = tid + split * nthreads; idx < B * (kHeadDim / 2); idx += nthreads * splits) {
                 int i = idx / (kHeadDim / 2), c = idx % (kHeadDim / 2);
@@ -316,7 +318,7 @@ int mma_splits(const goose_ctx* c, int S, int H) {
 }
 
 cudaError_t launch_tree_attn_mma(goose_ctx* c, const __nv_bfloat16* q, const __nv_bfloat16* kc,
-                                 const __nv_bfloat16* vc, const int64_t* row_off, const int32_t* ctx_len,
+                                 const __nv_bfloat16* vc, int64_t kv_rows, const int64_t* row_off, const int32_t* ctx_len,
                                  const int32_t* parent, int S, int B, int H, float scale,
                                  __nv_bfloat16* out, float* lse, cudaStream_t st) {
     if (S == 0 || H == 0) return cudaSuccess;
@@ -325,7 +327,7 @@ cudaError_t launch_tree_attn_mma(goose_ctx* c, const __nv_bfloat16* q, const __n
     if (warps < 4) warps = 4;
     dim3 grid(splits, H, S);
     cudaError_t e = launch_pdl(tree_attn_mma_kernel, grid, dim3(warps * 32), kMmaSmem, st, q, kc, vc, row_off, ctx_len,
-                               parent, B, H, scale * kLog2e, splits, c->partials, c->head_counters, c->status, out, lse);
+                               parent, B, H, kv_rows, scale * kLog2e, splits, c->partials, c->head_counters, c->status, out, lse);
     c->launches++;
     return e;
 }

@@ -220,7 +220,8 @@ struct Work {
     int S, H, B, G;
     long long total;          // all items
     bool small;               // total * (G + 1) fits 31 bits: 32-bit arithmetic (64-bit division is slow on the GPU)
-    __device__ __forceinline__ int tiles(int s) const { return (ctx_len[s] + B + kTile - 1) / kTile; }
+    // ctx_len comes from device memory: a negative value is treated as 0 (the tree rows alone)
+    __device__ __forceinline__ int tiles(int s) const { return (max(ctx_len[s], 0) + B + kTile - 1) / kTile; }
     __device__ __forceinline__ void init() {
         long long tot = 0;
         for (int s = 0; s < S; ++s) tot += (long long)H * tiles(s);
@@ -271,7 +272,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                       const __grid_constant__ CUtensorMap tmap_v, const int64_t* __restrict__ row_off,
                       const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ parent,
-                      int S, int B, int H, float scale_log2, float* __restrict__ partials,
+                      int S, int B, int H, int64_t kv_rows, float scale_log2, float* __restrict__ partials,
                       int32_t* __restrict__ status,
                       __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
     extern __shared__ unsigned char smem_raw[];
@@ -451,7 +452,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
 
             while (ok && cu.w < w_end) {
                 const int s0 = cu.s, h0 = cu.h, T = cu.T;
-                const int ctx = ctx_len[s0];
+                const int ctx = max(ctx_len[s0], 0);
                 const int n_keys = ctx + B;
                 const int32_t* par = parent + (size_t)s0 * B;
                 const int t_first = cu.t;
@@ -464,11 +465,16 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                         hd->par[row] = p;
                         if ((row == 0) ? (p != -1) : (p < 0 || p >= row)) hd->bad_parent = 1;
                     }
+                    // the sequence's rows must lie inside the cache (TMA would only read zeros outside, but the
+                    // result would be meaningless): treated like an invalid tree, with its own status bit
+                    const int64_t r0 = row_off[s0];
+                    const bool bad_rows = ctx_len[s0] < 0 || r0 < 0 || r0 + ctx + B > kv_rows;
+                    if (bad_rows && sm_tid == 0) { hd->bad_parent = 1; atomicOr(&status[s0], GOOSE_ST_BAD_ROWS); }
                     ok = group_sync(hd, gsync, status);
                     bad = hd->bad_parent != 0;
                     ok = ok && group_sync(hd, gsync, status);
                     if (!ok) break;
-                    if (sm_tid == 0 && bad) { hd->bad_parent = 0; atomicOr(&status[s0], GOOSE_ST_BAD_PARENT); }
+                    if (sm_tid == 0 && bad) { hd->bad_parent = 0; if (!bad_rows) atomicOr(&status[s0], GOOSE_ST_BAD_PARENT); }
                     anc[0] = anc[1] = anc[2] = anc[3] = 0;
                     if (row < B) {
                         if (bad) {
@@ -841,7 +847,7 @@ cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __
     int grid = c->num_sms;
     if (2 * grid > c->n_slots) grid = c->n_slots / 2;
     cudaError_t e = launch_pdl(tree_attn_umma_kernel, dim3(grid), dim3(kThreads), kUmmaSmem, st, mq, mk, mv, row_off,
-                               ctx_len, parent, S, B, H, scale * kLog2e, c->partials, c->status, out, lse);
+                               ctx_len, parent, S, B, H, kv_rows, scale * kLog2e, c->partials, c->status, out, lse);
     c->launches++;
     if (e != cudaSuccess) return e;
 #ifdef GOOSE_TRACE

@@ -255,6 +255,36 @@ def test_kv_compact_invalid_path_is_flagged(goose):
     assert np.array_equal(binding.bf16_to_bits(d["k_cache"])[:18], before[:18])   # sequence 0 untouched
 
 
+def test_rows_outside_the_cache_are_flagged_and_nothing_is_moved(goose):
+    """ctx_len / row_off are device data: a sequence whose rows would fall outside [0, kv_rows) is skipped."""
+    from paper_2604_02047_b200 import binding
+    x = synth.make_inputs(3, 2, 8, [10, 10, 10], [synth.chain_tree(8)] * 3, V=64, seed=4)
+    d = binding.to_device(x)
+    before_k = binding.bf16_to_bits(d["k_cache"]).copy()
+    bad_ctx = torch.tensor([10, -5, 10], dtype=torch.int32).cuda()
+    bad_off = torch.tensor([0, 18, 1 << 40], dtype=torch.int64).cuda()        # sequence 2 far outside the buffer
+    path = torch.tensor([[0, 2, 3, -1, -1, -1, -1, -1]] * 3, dtype=torch.int32).cuda()
+    alen = torch.tensor([2, 2, 2], dtype=torch.int32).cuda()
+    goose.kv_compact(d["k_cache"], d["v_cache"], bad_off, bad_ctx, path, alen)
+    assert goose.last_status(3).tolist() == [0, 8, 8]
+    after_k = binding.bf16_to_bits(d["k_cache"])
+    assert np.array_equal(after_k[18:], before_k[18:]) and not np.array_equal(after_k[:18], before_k[:18])
+    o = goose.verify_step(d["q"], d["k_cache"], d["v_cache"], bad_off, bad_ctx, d["parent"], d["draft_tok"],
+                          d["logits"], 4, x.scale)
+    torch.cuda.synchronize()
+    assert goose.last_status(3).tolist() == [0, 8, 8]                         # no fault, the step completes
+    got = o["out"].float().cpu().numpy()
+    assert np.all(got[1:] == 0) and np.abs(got[0]).max() > 0                   # flagged sequences: zero-filled output
+    for impl in _impls():                                                      # both attention kernels, same verdict
+        goose.set_attn_impl(impl)
+        try:
+            out, _ = goose.tree_attn(d["q"], d["k_cache"], d["v_cache"], bad_off, bad_ctx, d["parent"], x.scale)
+            torch.cuda.synchronize()
+        finally:
+            goose.set_attn_impl(binding.ATTN_AUTO)
+        assert goose.last_status(3).tolist() == [0, 8, 8] and torch.all(out[1:] == 0)
+
+
 # ------------------------------------------------------------------ whole step on the benchmark configs
 def _check_step(goose, oracle, x, n_rows=192, host=False):
     from paper_2604_02047_b200 import binding

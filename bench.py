@@ -191,7 +191,9 @@ def run_ours(args, x, cfg, rank, world, local_rank):
     import torch
     from paper_2604_02047_b200 import binding, build, synth
 
-    build.build()
+    if local_rank == 0:                  # one builder per node (a no-op when the shipped library matches the sources)
+        build.build()
+    dist_barrier()
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     g = binding.Goose(max_S=x.S, max_B=128, max_H=max(64, x.H), device=local_rank)

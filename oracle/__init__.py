@@ -21,13 +21,17 @@ _lib: Optional[ctypes.CDLL] = None
 
 def build(force: bool = False) -> str:
     """Compile the oracle if the shared object is missing or older than its source."""
-    if (not force and os.path.exists(_LIB)
-            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+    import hashlib
+    src_hash = hashlib.sha256(open(_SRC, "rb").read()).hexdigest()
+    hash_file = _LIB + ".srchash"
+    if not force and os.path.exists(_LIB) and os.path.exists(hash_file) and open(hash_file).read().strip() == src_hash:
         return _LIB
     tmp = _LIB + ".tmp%d" % os.getpid()
     cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c99", "-o", tmp, _SRC, "-lm"]
     subprocess.run(cmd, check=True, capture_output=True)
     os.replace(tmp, _LIB)
+    with open(hash_file, "w") as f:
+        f.write(src_hash + "\n")
     return _LIB
 
 

@@ -21,14 +21,25 @@ def _nvcc() -> str:
     return cand if os.path.exists(cand) else "nvcc"
 
 
-def _deps_mtime() -> float:
-    files = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(INCLUDE, "goose.h"), __file__]
-    return max(os.path.getmtime(f) for f in files)
+HASH_FILE = LIB + ".srchash"
+
+
+def _source_hash() -> str:
+    """Hash of everything the library is built from (contents, not time stamps: a copied tree keeps no mtimes)."""
+    import hashlib
+    h = hashlib.sha256()
+    files = sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC)) + [os.path.join(INCLUDE, "goose.h")]
+    for f in files:
+        h.update(os.path.basename(f).encode())
+        h.update(open(f, "rb").read())
+    h.update(" ".join(NVCC_FLAGS + SOURCES).encode())
+    return h.hexdigest()
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu for sm_100a and link libgoose.so; no-op when it is up to date."""
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _deps_mtime():
+    """Compile every source for sm_100a and link libgoose.so; no-op when the library matches the sources."""
+    src_hash = _source_hash()
+    if not force and os.path.exists(LIB) and os.path.exists(HASH_FILE) and open(HASH_FILE).read().strip() == src_hash:
         return LIB
     objdir = os.path.join(HERE, "build")
     os.makedirs(objdir, exist_ok=True)
@@ -54,6 +65,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         sys.stderr.write(r.stdout + r.stderr)
         raise RuntimeError("link failed")
     os.replace(tmp, LIB)
+    with open(HASH_FILE, "w") as f:
+        f.write(src_hash + "\n")
     return LIB
 
 

@@ -32,13 +32,12 @@ namespace goose {
 namespace {
 
 constexpr int kTile = 128;                      // keys per tile
-constexpr int kStages = 4;                      // ring of K/V stages
+constexpr int kStages = 5;                      // ring of K/V stages (P lives in tensor memory, not here)
 constexpr int kStageBytes = kTile * kHeadDim * 2;   // 32 KB: one K or one V tile
 constexpr int kHalfBytes = kTile * 128;         // 16 KB: 128 rows x 64 bf16 (one swizzle-atom column)
 constexpr int kQBytes = 2 * kHalfBytes;
-constexpr int kPBytes = 2 * kHalfBytes;
 constexpr int kHeaderBytes = 1024;
-constexpr int kUmmaSmem = kHeaderBytes + 1024 /*alignment slack*/ + 2 * kQBytes + kPBytes + kStages * kStageBytes;
+constexpr int kUmmaSmem = kHeaderBytes + 1024 /*alignment slack*/ + 2 * kQBytes + kStages * kStageBytes;
 constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;
@@ -165,6 +164,12 @@ __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint6
                  "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                  ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
 }
+// same, with the A operand (M x 16 bf16, two per 32-bit column, lane = row) read from tensor memory
+__device__ __forceinline__ void umma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
 __device__ __forceinline__ void umma_commit(unsigned long long* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -280,8 +285,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     unsigned char* buf = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + kHeaderBytes + 1023) & ~(uintptr_t)1023);
     unsigned char* q_smem = buf;
-    unsigned char* p_smem = buf + 2 * kQBytes;
-    unsigned char* kv_smem = buf + 2 * kQBytes + kPBytes;
+    unsigned char* kv_smem = buf + 2 * kQBytes;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -378,11 +382,11 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 bool ok = true;
                 TRACE_DECL;
                 TRACE(1, tn, 1);
-                const uint32_t q_base = smem_u32(q_smem), p_addr = smem_u32(p_smem), kv_addr = smem_u32(kv_smem);
+                const uint32_t q_base = smem_u32(q_smem), kv_addr = smem_u32(kv_smem);
                 constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
 
                 auto issue_pv = [&](uint32_t j, bool first_of_segment) -> bool {
-                    // tile j's P is in shared memory and S(j) has been consumed
+                    // tile j's P (bf16) has replaced S(j) in the first 64 columns of its S buffer
                     if (!mbar_wait(hd, &hd->p_ready, j & 1, status)) return false;
                     const uint32_t ring = 2 * j + 1, st = ring % kStages;
                     if (!mbar_wait(hd, &hd->kv_full[st], (ring / kStages) & 1, status)) return false;
@@ -392,9 +396,9 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                     const uint32_t v_addr = kv_addr + st * kStageBytes;
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {       // 16 keys per instruction
-                        uint64_t a = smem_desc(p_addr + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16, 1024);
                         uint64_t b = smem_desc(v_addr + kk * 2048, kHalfBytes, 1024);   // MN-major: LBO = next 64 d
-                        umma_f16(tmem + kColO, a, b, idesc_pv, (!first_of_segment || kk > 0) ? 1u : 0u);
+                        umma_f16_ts(tmem + kColO, tmem + kColS + (j & 1) * 128 + kk * 8, b, idesc_pv,
+                                    (!first_of_segment || kk > 0) ? 1u : 0u);
                     }
                     umma_commit(&hd->kv_empty[st]);
                     umma_commit(&hd->pv_done);
@@ -563,29 +567,28 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                         }
                         m_use = (m_run == -INFINITY) ? 0.f : m_run;
                     }
-                    // P(jg) may overwrite P(jg-1) only after PV(jg-1) has read it
-                    if (ok && jg > 0) ok = mbar_wait(hd, &hd->pv_done, (jg - 1) & 1, status);
-                    if (!ok) break;
+                    // P (bf16 pairs) overwrites the first 64 columns of this tile's S buffer: this thread has its whole
+                    // S row in registers, and QK^T of tile jg+2 is ordered after PV(jg) in the MMA pipe
                     if (warp_has_rows) {
                         float ls4[4] = {0.f, 0.f, 0.f, 0.f};
                         const float neg_m = -m_use;
-                        unsigned char* prow = p_smem + row * 128;
 #pragma unroll
-                        for (int ch = 0; ch < 16; ++ch) {  // 16-byte chunks of 8 keys
-                            uint32_t pk[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                float p0 = ex2(fmaf(__uint_as_float(v[ch * 8 + 2 * e]), scale_log2, neg_m));
-                                float p1 = ex2(fmaf(__uint_as_float(v[ch * 8 + 2 * e + 1]), scale_log2, neg_m));
-                                ls4[e] += p0 + p1;
-                                pk[e] = pack_bf16x2(p0, p1);
-                            }
-                            const int half = ch >> 3, cin = ch & 7;
-                            *reinterpret_cast<uint4*>(prow + half * kHalfBytes + ((cin ^ (row & 7)) << 4)) =
-                                make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        for (int e = 0; e < 64; ++e) {
+                            float p0 = ex2(fmaf(__uint_as_float(v[2 * e]), scale_log2, neg_m));
+                            float p1 = ex2(fmaf(__uint_as_float(v[2 * e + 1]), scale_log2, neg_m));
+                            ls4[e & 3] += p0 + p1;
+                            v[e] = pack_bf16x2(p0, p1);
                         }
                         l_run += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+                        const uint32_t p_taddr = tmem + kColS + (jg & 1) * 128 + lane_sel;
+                        TMEM_ST32(p_taddr, v, 0);
+                        TMEM_ST32(p_taddr + 32, v, 32);
+                        tmem_wait_st();
                     }
+                    // observe every phase of pv_done in order (a parity wait must never lag two phases behind its
+                    // barrier); by now PV(jg-1) has normally completed, so this does not stall
+                    if (jg > 0) ok = mbar_wait(hd, &hd->pv_done, (jg - 1) & 1, status);
+                    if (!ok) break;
                     // ragged end: V rows past the sequence's last key may hold anything -> zero them
                     if ((t + 1) * kTile > n_keys) {
                         const uint32_t ring = 2 * jg + 1, st = ring % kStages;
@@ -600,8 +603,8 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                                 *reinterpret_cast<uint4*>(vrow + kHalfBytes + c * 16) = make_uint4(0, 0, 0, 0);
                             }
                         }
+                        fence_proxy_async();               // generic-proxy writes -> visible to the tensor core
                     }
-                    fence_proxy_async();                   // generic-proxy writes -> visible to the tensor core
                     tc_fence_before();
                     mbar_arrive(&hd->p_ready);
                     if (sm_tid == 0 && seg_tiles < 2) TRACE(2, tn, 3);

@@ -33,8 +33,8 @@ UNIT = "steps/s"
 L2_BYTES = 126 * 1024 * 1024
 # DRAM traffic per attention launch from the ncu capture summarised under profiles/ (bytes), per config
 # name; None = not captured for that workload.
-NCU_TRAFFIC_BYTES = {"33b": 227_392_000,    # tree_attn_umma_kernel: 223.29 MB read + 4.1 MB written per launch
-                     "13b": 89_430_000}     # 86.42 MB read + 3.0 MB written
+NCU_TRAFFIC_BYTES = {"33b": 227_470_000,    # tree_attn_umma_kernel: 223.29 MB read + 4.2 MB written per launch
+                     "13b": 89_450_000}     # 86.42 MB read + 3.0 MB written
 
 
 def _peaks():

@@ -698,8 +698,9 @@ tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, int S, int B, int 
                          float* __restrict__ lse) {
     const int rg = blockIdx.x, h = blockIdx.y, s = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    pdl_wait();                                            // the main kernel's partials are complete and visible
-    pdl_trigger();
+    // The partition arithmetic needs only ctx_len[], which is final before this kernel's CTAs can start: the main
+    // kernel triggers its dependents after its own pdl_wait(), i.e. after whatever produced ctx_len[] completed.
+    // So all of it runs before the wait, and the partial loads are issued the moment the main grid is done.
     Work wk;
     wk.ctx_len = ctx_len; wk.S = S; wk.H = H; wk.B = B; wk.G = G;
     wk.init();
@@ -708,13 +709,17 @@ tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, int S, int B, int 
     const int T = wk.tiles(s);
     const long long head_first = off + (long long)h * T;
     const int c_lo = wk.cta_of(head_first), c_hi = wk.cta_of(head_first + T - 1);
-    if (c_lo == c_hi) return;                              // written directly by the main kernel
+    const bool whole = c_lo == c_hi;                       // written directly by the main kernel
     const int row = rg * 32 + lane;
-    if (row >= B) return;
     // CTA c's partial for this head sits in slot 2c, or 2c+1 when its segment starts at the head's first tile,
     // which only the first CTA can do.  With fewer items than CTAs some CTAs in [c_lo, c_hi] are empty.
     const int flag_lo = wk.cta_start(c_lo) <= head_first ? 1 : 0;
     const bool sparse = wk.total < G;
+    // every CTA waits, also those with nothing to do: the next kernel in the stream relies on "this grid is
+    // complete" implying "the main grid is complete"
+    pdl_wait();                                            // the main kernel's partials are complete and visible
+    pdl_trigger();
+    if (whole || row >= B) return;
     float M_run = -INFINITY, L_run = 0.f;
     float acc[16];                                         // warp w owns columns 16w .. 16w+15 (column groups 2w, 2w+1)
 #pragma unroll

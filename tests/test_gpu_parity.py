@@ -91,6 +91,23 @@ def test_attention_ragged_batch_and_peaked_scores(goose, oracle, impl):
 
 
 @pytest.mark.parametrize("impl", _impls(), ids=_impl_ids())
+def test_attention_extreme_partitions(goose, oracle, impl):
+    """One head split over every CTA (about 150 partials to merge), and many tiny sequences (fewer items than CTAs
+    per head boundary, CTAs that own several whole heads)."""
+    x = synth.make_inputs(1, 1, 8, [40000], [synth.kary_tree(8, 2)], V=8, with_logits=False, seed=41)
+    out, lse, st = _run_attn(goose, x, impl)
+    ss, si, sh = np.zeros(8, np.int32), np.arange(8, dtype=np.int32), np.zeros(8, np.int32)
+    ref, ref_lse = oracle.tree_attn_rows(x.q, x.k_cache, x.v_cache, x.row_off, x.ctx_len, x.parent, x.scale, ss, si, sh)
+    assert not st.any() and attn_row_err(out[0, :, 0], ref).max() <= ATTN_TOL
+    assert np.abs(lse[0, :, 0] - ref_lse).max() <= 2e-3
+    rng = np.random.default_rng(43)
+    S = 16
+    y = synth.make_inputs(S, 12, 5, rng.integers(0, 300, S), [synth.random_tree(rng, 5) for _ in range(S)], V=8,
+                          with_logits=False, seed=44)
+    _check_attn_full(goose, oracle, y, impl)
+
+
+@pytest.mark.parametrize("impl", _impls(), ids=_impl_ids())
 def test_attention_never_reads_rows_past_the_tree(goose, oracle, impl):
     """Rows behind ctx+B (slack, or another sequence's rows) may hold anything, NaN included."""
     from paper_2604_02047_b200 import binding

@@ -47,7 +47,8 @@ def lib() -> ctypes.CDLL:
         build()
         _lib = ctypes.CDLL(_LIB)
         _lib.oracle_num_threads.restype = ctypes.c_int
-        for name in ("oracle_tree_attn", "oracle_tree_attn_rows", "oracle_node_topk", "oracle_accept",
+        for name in ("oracle_tree_attn", "oracle_tree_attn_rows", "oracle_tree_attn_gqa", "oracle_tree_attn_rows_gqa",
+                     "oracle_node_topk", "oracle_accept",
                      "oracle_kv_compact", "oracle_check_parent", "oracle_harvest"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
@@ -64,17 +65,22 @@ def _c(a, dt) -> np.ndarray:
 
 def tree_attn(q, k_cache, v_cache, row_off, ctx_len, parent, scale: float, want_lse: bool = True
               ) -> Tuple[np.ndarray, Optional[np.ndarray]]:
-    """q uint16 [S][B][H][D]; caches uint16 [rows][H][D].  Returns out fp64 [S][B][H][D], lse [S][B][H]."""
+    """q uint16 [S][B][H][D]; caches uint16 [rows][Hkv][D] (Hkv == H: multi-head attention; Hkv a divisor of H:
+    grouped-query attention, query head h reads key/value head h // (H // Hkv)).
+    Returns out fp64 [S][B][H][D], lse [S][B][H]."""
     q = _c(q, np.uint16); k_cache = _c(k_cache, np.uint16); v_cache = _c(v_cache, np.uint16)
     S, B, H, D = q.shape
+    Hkv = k_cache.shape[1]
+    if v_cache.shape != k_cache.shape or k_cache.shape[2] != D or Hkv < 1 or H % Hkv != 0:
+        raise ValueError("cache shape %r does not fit q shape %r" % (k_cache.shape, q.shape))
     row_off = _c(row_off, np.int64).reshape(S); ctx_len = _c(ctx_len, np.int32).reshape(S)
     parent = _c(parent, np.int32).reshape(S, B)
     out = np.zeros((S, B, H, D), dtype=np.float64)
     lse = np.zeros((S, B, H), dtype=np.float64) if want_lse else None
-    rc = lib().oracle_tree_attn(_ptr(q, ctypes.c_uint16), _ptr(k_cache, ctypes.c_uint16), _ptr(v_cache, ctypes.c_uint16),
-                                _ptr(row_off, ctypes.c_int64), _ptr(ctx_len, ctypes.c_int32), _ptr(parent, ctypes.c_int32),
-                                ctypes.c_int(S), ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(D),
-                                ctypes.c_double(scale), _ptr(out, ctypes.c_double), _ptr(lse, ctypes.c_double))
+    rc = lib().oracle_tree_attn_gqa(_ptr(q, ctypes.c_uint16), _ptr(k_cache, ctypes.c_uint16), _ptr(v_cache, ctypes.c_uint16),
+                                    _ptr(row_off, ctypes.c_int64), _ptr(ctx_len, ctypes.c_int32), _ptr(parent, ctypes.c_int32),
+                                    ctypes.c_int(S), ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D),
+                                    ctypes.c_double(scale), _ptr(out, ctypes.c_double), _ptr(lse, ctypes.c_double))
     if rc != 0:
         raise ValueError("oracle_tree_attn failed: rc=%d (invalid parent[]?)" % rc)
     return out, lse
@@ -82,18 +88,21 @@ def tree_attn(q, k_cache, v_cache, row_off, ctx_len, parent, scale: float, want_
 
 def tree_attn_rows(q, k_cache, v_cache, row_off, ctx_len, parent, scale: float, ss, si, sh
                    ) -> Tuple[np.ndarray, np.ndarray]:
-    """Same as :func:`tree_attn` for sampled (sequence, node, head) rows only."""
+    """Same as :func:`tree_attn` for sampled (sequence, node, query head) rows only."""
     q = _c(q, np.uint16); k_cache = _c(k_cache, np.uint16); v_cache = _c(v_cache, np.uint16)
     S, B, H, D = q.shape
+    Hkv = k_cache.shape[1]
+    if v_cache.shape != k_cache.shape or k_cache.shape[2] != D or Hkv < 1 or H % Hkv != 0:
+        raise ValueError("cache shape %r does not fit q shape %r" % (k_cache.shape, q.shape))
     row_off = _c(row_off, np.int64).reshape(S); ctx_len = _c(ctx_len, np.int32).reshape(S)
     parent = _c(parent, np.int32).reshape(S, B)
     ss = _c(ss, np.int32); si = _c(si, np.int32); sh = _c(sh, np.int32)
     n = len(ss)
     out = np.zeros((n, D), dtype=np.float64)
     lse = np.zeros((n,), dtype=np.float64)
-    rc = lib().oracle_tree_attn_rows(_ptr(q, ctypes.c_uint16), _ptr(k_cache, ctypes.c_uint16), _ptr(v_cache, ctypes.c_uint16),
+    rc = lib().oracle_tree_attn_rows_gqa(_ptr(q, ctypes.c_uint16), _ptr(k_cache, ctypes.c_uint16), _ptr(v_cache, ctypes.c_uint16),
                                      _ptr(row_off, ctypes.c_int64), _ptr(ctx_len, ctypes.c_int32), _ptr(parent, ctypes.c_int32),
-                                     ctypes.c_int(S), ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(D),
+                                     ctypes.c_int(S), ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D),
                                      ctypes.c_double(scale), ctypes.c_int(n), _ptr(ss, ctypes.c_int32),
                                      _ptr(si, ctypes.c_int32), _ptr(sh, ctypes.c_int32),
                                      _ptr(out, ctypes.c_double), _ptr(lse, ctypes.c_double))

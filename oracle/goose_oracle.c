@@ -74,13 +74,18 @@ int oracle_check_parent(const int32_t* parent, int B) {
 }
 
 /* ------------------------------------------------------------------ tree attention, one row
- * Node i of sequence s, head h.  Visible keys: prefix rows 0..ctx-1 and tree rows ctx+j, j in A(i).
+ * Node i of sequence s, query head h.  Visible keys: prefix rows 0..ctx-1 and tree rows ctx+j, j in A(i).
  *   s_j = scale * sum_d q[d] K[j][d];  p_j = exp(s_j - max) / sum exp(s - max);  out = sum_j p_j V[j].
- * K/V layout: [row][H][D], sequence s owns rows row_off[s] .. row_off[s]+ctx+B-1. */
+ * K/V layout: [row][Hkv][D], sequence s owns rows row_off[s] .. row_off[s]+ctx+B-1.
+ * Grouped-query attention (the 8B models of the paper's evaluation, Sec. 5 set-up, have 32 query heads over 8
+ * key/value heads): the H query heads are split into Hkv groups of H/Hkv consecutive heads, and every head of a
+ * group reads key/value head hk = h / (H/Hkv).  Hkv == H is ordinary multi-head attention (hk = h). */
 static int attn_row(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, int64_t row0, int ctx,
-                    const int32_t* parent, int B, int H, int D, double scale, int i, int h,
+                    const int32_t* parent, int B, int H, int Hkv, int D, double scale, int i, int h,
                     const uint16_t* qrow /* q[s][i][h][:] */, double* out /* [D] */, double* lse) {
     (void)q;
+    if (Hkv < 1 || H % Hkv != 0) return -3;
+    const int hk = h / (H / Hkv);
     int n = ctx + B;
     unsigned char* vis = (unsigned char*)malloc((size_t)B);
     double* sc = (double*)malloc(sizeof(double) * (size_t)n);
@@ -91,7 +96,7 @@ static int attn_row(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, i
     for (int j = 0; j < n; ++j) {
         int visible = (j < ctx) ? 1 : vis[j - ctx];
         if (!visible) { sc[j] = -INFINITY; continue; }
-        const uint16_t* krow = kc + ((size_t)(row0 + j) * H + h) * D;
+        const uint16_t* krow = kc + ((size_t)(row0 + j) * Hkv + hk) * D;
         double acc = 0.0;
         for (int d = 0; d < D; ++d) acc += bf16_to_f64(qrow[d]) * bf16_to_f64(krow[d]);
         sc[j] = scale * acc;
@@ -104,7 +109,7 @@ static int attn_row(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, i
     for (int j = 0; j < n; ++j) {
         if (sc[j] == -INFINITY) continue;
         double p = exp(sc[j] - mx) / denom;
-        const uint16_t* vrow = vc + ((size_t)(row0 + j) * H + h) * D;
+        const uint16_t* vrow = vc + ((size_t)(row0 + j) * Hkv + hk) * D;
         for (int d = 0; d < D; ++d) out[d] += p * bf16_to_f64(vrow[d]);
     }
     if (lse) *lse = mx + log(denom);
@@ -113,10 +118,11 @@ static int attn_row(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, i
     return 0;
 }
 
-/* Full output: out fp64 [S][B][H][D], lse fp64 [S][B][H] (may be NULL). Returns 0 or <0. */
-int oracle_tree_attn(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, const int64_t* row_off,
-                     const int32_t* ctx_len, const int32_t* parent, int S, int B, int H, int D,
-                     double scale, double* out, double* lse) {
+/* Full output: out fp64 [S][B][H][D], lse fp64 [S][B][H] (may be NULL). Returns 0 or <0.
+ * q has H heads, the caches Hkv heads (H a multiple of Hkv). */
+int oracle_tree_attn_gqa(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, const int64_t* row_off,
+                         const int32_t* ctx_len, const int32_t* parent, int S, int B, int H, int Hkv, int D,
+                         double scale, double* out, double* lse) {
     int rc = 0;
     long total = (long)S * B * H;
 #pragma omp parallel for schedule(dynamic, 4)
@@ -125,7 +131,7 @@ int oracle_tree_attn(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, 
         int i = (int)((t / H) % B);
         int s = (int)(t / ((long)H * B));
         const uint16_t* qrow = q + (((size_t)s * B + i) * H + h) * D;
-        int r = attn_row(q, kc, vc, row_off[s], ctx_len[s], parent + (size_t)s * B, B, H, D, scale, i, h, qrow,
+        int r = attn_row(q, kc, vc, row_off[s], ctx_len[s], parent + (size_t)s * B, B, H, Hkv, D, scale, i, h, qrow,
                          out + (size_t)t * D, lse ? lse + t : NULL);
         if (r != 0) {
 #pragma omp critical
@@ -135,18 +141,24 @@ int oracle_tree_attn(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, 
     return rc;
 }
 
+int oracle_tree_attn(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, const int64_t* row_off,
+                     const int32_t* ctx_len, const int32_t* parent, int S, int B, int H, int D,
+                     double scale, double* out, double* lse) {
+    return oracle_tree_attn_gqa(q, kc, vc, row_off, ctx_len, parent, S, B, H, H, D, scale, out, lse);
+}
+
 /* Sampled rows: for each sample n the row (s,i,h) = (ss[n], si[n], sh[n]); out [n][D], lse [n]. */
-int oracle_tree_attn_rows(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, const int64_t* row_off,
-                          const int32_t* ctx_len, const int32_t* parent, int S, int B, int H, int D,
-                          double scale, int n_samples, const int32_t* ss, const int32_t* si,
-                          const int32_t* sh, double* out, double* lse) {
+int oracle_tree_attn_rows_gqa(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, const int64_t* row_off,
+                              const int32_t* ctx_len, const int32_t* parent, int S, int B, int H, int Hkv, int D,
+                              double scale, int n_samples, const int32_t* ss, const int32_t* si,
+                              const int32_t* sh, double* out, double* lse) {
     int rc = 0;
     (void)S;
 #pragma omp parallel for schedule(dynamic, 1)
     for (int n = 0; n < n_samples; ++n) {
         int s = ss[n], i = si[n], h = sh[n];
         const uint16_t* qrow = q + (((size_t)s * B + i) * H + h) * D;
-        int r = attn_row(q, kc, vc, row_off[s], ctx_len[s], parent + (size_t)s * B, B, H, D, scale, i, h, qrow,
+        int r = attn_row(q, kc, vc, row_off[s], ctx_len[s], parent + (size_t)s * B, B, H, Hkv, D, scale, i, h, qrow,
                          out + (size_t)n * D, lse ? lse + n : NULL);
         if (r != 0) {
 #pragma omp critical
@@ -154,6 +166,14 @@ int oracle_tree_attn_rows(const uint16_t* q, const uint16_t* kc, const uint16_t*
         }
     }
     return rc;
+}
+
+int oracle_tree_attn_rows(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, const int64_t* row_off,
+                          const int32_t* ctx_len, const int32_t* parent, int S, int B, int H, int D,
+                          double scale, int n_samples, const int32_t* ss, const int32_t* si,
+                          const int32_t* sh, double* out, double* lse) {
+    return oracle_tree_attn_rows_gqa(q, kc, vc, row_off, ctx_len, parent, S, B, H, H, D, scale, n_samples, ss, si, sh,
+                                     out, lse);
 }
 
 /* ------------------------------------------------------------------ per-node argmax + top-k

@@ -33,7 +33,7 @@ class VerifyConfig:
 
     name: str
     S: int                      # sequences in the batch
-    H: int                      # attention heads (MHA: K/V heads == Q heads)
+    H: int                      # query heads
     B: int                      # tree nodes per sequence, root included
     ctx: Tuple[int, int]        # prefix length range [lo, hi] (lo == hi: fixed)
     spine: Tuple[int, int]      # spine node count incl. root, range [lo, hi]
@@ -43,6 +43,7 @@ class VerifyConfig:
     V: int = VOCAB
     k: int = 8
     D: int = HEAD_DIM
+    Hkv: Optional[int] = None   # key/value heads (None: multi-head attention, one per query head)
 
 
 CONFIGS: List[VerifyConfig] = [
@@ -56,6 +57,10 @@ CONFIGS: List[VerifyConfig] = [
                  p_spine=(0.8, 0.8), p_branch=0.15),
     VerifyConfig("batch16", S=16, H=32, B=64, ctx=(1024, 16384), spine=(4, 20), branch_len_max=3,
                  p_spine=(0.5, 0.95), p_branch=0.15),
+    # second workload: grouped-query attention and a large vocabulary, the shape of the 8B models of the
+    # paper's evaluation (32 query heads over 8 key/value heads, 128 256 vocabulary entries)
+    VerifyConfig("gqa8b", S=4, H=32, B=32, ctx=(4096, 16384), spine=(6, 12), branch_len_max=3,
+                 p_spine=(0.5, 0.95), p_branch=0.15, V=128256, Hkv=8),
 ]
 
 # stream ids: one independent generator per tensor
@@ -191,8 +196,8 @@ class VerifyInputs:
     k: int
     scale: float                       # 1/sqrt(D), python float (fp64)
     q: np.ndarray                      # uint16 [S][B][H][D]
-    k_cache: np.ndarray                # uint16 [rows][H][D]
-    v_cache: np.ndarray                # uint16 [rows][H][D]
+    k_cache: np.ndarray                # uint16 [rows][Hkv][D]
+    v_cache: np.ndarray                # uint16 [rows][Hkv][D]
     row_off: np.ndarray                # int64 [S]
     ctx_len: np.ndarray                # int32 [S]
     parent: np.ndarray                 # int32 [S][B]
@@ -209,12 +214,20 @@ class VerifyInputs:
     def kv_rows(self) -> int:
         return int(self.k_cache.shape[0])
 
+    @property
+    def Hkv(self) -> int:
+        return int(self.k_cache.shape[1])
+
 
 def make_inputs(S: int, H: int, B: int, ctx_lens, parents, *, V: int = VOCAB, k: int = 8,
                 seed: int = 0, config_id: int = 99, is_spine=None, p_spine=0.8, p_branch=0.15,
                 D: int = HEAD_DIM, with_logits: bool = True, q_gain: float = 1.0,
-                name: str = "custom") -> VerifyInputs:
-    """Build a step's inputs from explicit prefix lengths and parent arrays."""
+                name: str = "custom", Hkv: Optional[int] = None) -> VerifyInputs:
+    """Build a step's inputs from explicit prefix lengths and parent arrays.  ``Hkv`` key/value heads
+    (default: H, multi-head attention)."""
+    Hkv = H if Hkv is None else int(Hkv)
+    if Hkv < 1 or H % Hkv != 0:
+        raise ValueError("H must be a multiple of Hkv")
     ctx_lens = np.asarray(ctx_lens, dtype=np.int32).reshape(S)
     parents = np.asarray(parents, dtype=np.int32).reshape(S, B)
     if is_spine is None:
@@ -225,8 +238,8 @@ def make_inputs(S: int, H: int, B: int, ctx_lens, parents, *, V: int = VOCAB, k:
     row_off = np.concatenate([[0], np.cumsum(rows_per_seq)[:-1]]).astype(np.int64)
     total = int(rows_per_seq.sum())
     q = np.empty((S, B, H, D), dtype=np.uint16)
-    kc = np.empty((total, H, D), dtype=np.uint16)
-    vc = np.empty((total, H, D), dtype=np.uint16)
+    kc = np.empty((total, Hkv, D), dtype=np.uint16)
+    vc = np.empty((total, Hkv, D), dtype=np.uint16)
     tok = np.empty((S, B), dtype=np.int32)
     planted = np.zeros((S, B), dtype=bool)
     logits = np.empty((S * B, V), dtype=np.uint16) if with_logits else np.empty((0, V), dtype=np.uint16)
@@ -236,8 +249,8 @@ def make_inputs(S: int, H: int, B: int, ctx_lens, parents, *, V: int = VOCAB, k:
         if q_gain != 1.0:
             qf = qf * np.float32(q_gain)
         q[s] = f32_to_bf16_bits(qf)
-        kc[r0:r0 + n] = normal_bf16(_rng(seed, config_id, s, _ST_K), (n, H, D))
-        vc[r0:r0 + n] = normal_bf16(_rng(seed, config_id, s, _ST_V), (n, H, D))
+        kc[r0:r0 + n] = normal_bf16(_rng(seed, config_id, s, _ST_K), (n, Hkv, D))
+        vc[r0:r0 + n] = normal_bf16(_rng(seed, config_id, s, _ST_V), (n, Hkv, D))
         tok[s] = distinct_sibling_tokens(_rng(seed, config_id, s, _ST_TOK), parents[s], V if with_logits else max(V, 4096))
         if with_logits:
             bits, pl = planted_logits(_rng(seed, config_id, s, _ST_LOGIT), _rng(seed, config_id, s, _ST_PLANT),
@@ -266,20 +279,21 @@ def config_shapes(config_id: int, seed: int = 0):
 
 def make_config(config_id: int, seed: int = 0, *, with_logits: bool = True,
                 ctx_override: Optional[int] = None) -> VerifyInputs:
-    """Inputs of benchmark config ``config_id`` (0..4).  ``ctx_override`` shrinks the prefix
+    """Inputs of benchmark config ``config_id`` (0..5).  ``ctx_override`` shrinks the prefix
     (same tree / heads / vocabulary) for cases the oracle should finish quickly."""
     cfg, ctxs, parents, spines, ps = config_shapes(config_id, seed)
     if ctx_override is not None:
         ctxs = np.minimum(ctxs, np.int32(ctx_override))
     return make_inputs(cfg.S, cfg.H, cfg.B, ctxs, parents, V=cfg.V, k=cfg.k, seed=seed,
                        config_id=config_id, is_spine=spines, p_spine=ps, p_branch=cfg.p_branch,
-                       D=cfg.D, with_logits=with_logits, name=cfg.name)
+                       D=cfg.D, with_logits=with_logits, name=cfg.name, Hkv=cfg.Hkv)
 
 
-def algorithmic_bytes(S: int, H: int, B: int, D: int, V: int, ctx_lens) -> Dict[str, int]:
+def algorithmic_bytes(S: int, H: int, B: int, D: int, V: int, ctx_lens, Hkv: Optional[int] = None) -> Dict[str, int]:
     """Bytes each part of the step must move at least once (bf16 = 2 bytes)."""
     ctx_lens = np.asarray(ctx_lens, dtype=np.int64)
-    kv = int((2 * (ctx_lens + B) * H * D * 2).sum())
+    Hkv = H if Hkv is None else Hkv
+    kv = int((2 * (ctx_lens + B) * Hkv * D * 2).sum())
     qo = int(2 * S * B * H * D * 2)
     logits = int(S * B * V * 2)
     return {"attn": kv + qo, "topk": logits, "total": kv + qo + logits}

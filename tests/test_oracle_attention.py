@@ -149,3 +149,50 @@ def test_invalid_parent_is_rejected(oracle):
     with pytest.raises(ValueError):
         oracle.tree_attn(x.q, x.k_cache, x.v_cache, x.row_off, x.ctx_len, bad, x.scale)
     assert not oracle.check_parent(bad) and oracle.check_parent(x.parent)
+
+
+# ------------------------------------------------------------------ grouped-query attention
+def test_gqa_equals_mha_on_replicated_kv_heads(oracle):
+    """Query head h of a grouped-query model reads key/value head h // g (groups of g consecutive query heads):
+    the result is that of multi-head attention over caches whose heads are each repeated g times in place."""
+    for H, Hkv in ((8, 2), (6, 2), (4, 1), (3, 3)):
+        g = H // Hkv
+        x = _small(S=2, H=H, B=7, ctx=(19, 4), seed=5 + H, Hkv=Hkv)
+        assert x.k_cache.shape[1] == Hkv
+        out, lse = oracle.tree_attn(x.q, x.k_cache, x.v_cache, x.row_off, x.ctx_len, x.parent, x.scale)
+        k_rep, v_rep = np.repeat(x.k_cache, g, axis=1), np.repeat(x.v_cache, g, axis=1)
+        ref, ref_lse = oracle.tree_attn(x.q, k_rep, v_rep, x.row_off, x.ctx_len, x.parent, x.scale)
+        assert np.array_equal(out, ref) and np.array_equal(lse, ref_lse)
+        if g > 1 and Hkv > 1:
+            # the interleaved assignment (h % Hkv) is a different function
+            k_til, v_til = np.tile(x.k_cache, (1, g, 1)), np.tile(x.v_cache, (1, g, 1))
+            other, _ = oracle.tree_attn(x.q, k_til, v_til, x.row_off, x.ctx_len, x.parent, x.scale)
+            assert np.abs(other - ref).max() > 1e-3
+
+
+def test_gqa_rows_by_direct_formula(oracle):
+    """Every (node, query head) row written out with numpy: softmax over prefix + ancestors of the group's KV head."""
+    H, Hkv, B = 6, 3, 10
+    x = _small(S=1, H=H, B=B, ctx=(21,), seed=23, Hkv=Hkv)
+    out, lse = oracle.tree_attn(x.q, x.k_cache, x.v_cache, x.row_off, x.ctx_len, x.parent, x.scale)
+    K, V, Q = _f64(x.k_cache), _f64(x.v_cache), _f64(x.q)
+    for i in range(B):
+        chain, v = [], i
+        while v != -1:
+            chain.append(v); v = int(x.parent[0, v])
+        rows = list(range(21)) + [21 + j for j in sorted(chain)]
+        for h in range(H):
+            hk = h // (H // Hkv)
+            sc = (K[rows, hk, :] @ Q[0, i, h, :]) / np.sqrt(128.0)
+            assert np.abs(out[0, i, h] - softmax(sc) @ V[rows, hk, :]).max() < 1e-12
+            assert abs(lse[0, i, h] - logsumexp(sc)) < 1e-12
+    # sampled-row entry point agrees with the full one
+    ss = np.zeros(5, np.int32); si = np.array([0, 3, 9, 4, 7], np.int32); sh = np.array([5, 0, 2, 3, 4], np.int32)
+    o2, l2 = oracle.tree_attn_rows(x.q, x.k_cache, x.v_cache, x.row_off, x.ctx_len, x.parent, x.scale, ss, si, sh)
+    assert np.array_equal(o2, out[ss, si, sh]) and np.array_equal(l2, lse[ss, si, sh])
+
+
+def test_gqa_rejects_heads_that_do_not_divide(oracle):
+    x = _small(S=1, H=4, B=5, ctx=(8,), seed=2)
+    with pytest.raises(ValueError):
+        oracle.tree_attn(x.q, x.k_cache[:, :3], x.v_cache[:, :3], x.row_off, x.ctx_len, x.parent, x.scale)

@@ -176,7 +176,7 @@ def run_reference(args, x, cfg_name):
         "impl": "reference", "metric": METRIC, "value": 1.0 / step_s, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": cfg_name, "S": x.S, "H": x.H, "B": x.B, "V": x.V, "k": x.k,
+        "config": {"workload": cfg_name, "S": x.S, "H": x.H, "Hkv": x.Hkv, "B": x.B, "V": x.V, "k": x.k,
                    "note": "fp64 CPU oracle on a bounded sample per step, scaled to a whole step"},
         "cpu_baseline": {"value": 1.0 / step_s, "unit": UNIT, "cores": res["cores"], "kind": "oracle",
                          "sample": res["sample"]},
@@ -201,7 +201,11 @@ def run_ours(args, x, cfg, rank, world, local_rank):
         g.set_attn_impl({"mma": binding.ATTN_MMA, "umma": binding.ATTN_UMMA}[args.attn_impl])
 
     base = binding.to_device(x, dev)
-    ab = synth.algorithmic_bytes(x.S, x.H, x.B, x.D, x.V, x.ctx_len)
+    ab = synth.algorithmic_bytes(x.S, x.H, x.B, x.D, x.V, x.ctx_len, Hkv=x.Hkv)
+    gqa = x.Hkv != x.H          # grouped-query workload: the *_gqa entry points
+    verify_step = g.verify_step_gqa if gqa else g.verify_step
+    tree_attn = g.tree_attn_gqa if gqa else g.tree_attn
+    verify_step_host = g.verify_step_host_gqa if gqa else g.verify_step_host
     footprint = sum(t.numel() * t.element_size() for t in base.values())
     R = int(max(2, min(64, -(-max(2 * L2_BYTES, 1 << 30) // footprint))))
     reps = [base] + [{k: v.clone() for k, v in base.items()} for _ in range(R - 1)]
@@ -210,12 +214,12 @@ def run_ours(args, x, cfg, rank, world, local_rank):
 
     def step(i):
         d, o = reps[i % R], outs[i % R]
-        g.verify_step(d["q"], d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], d["parent"], d["draft_tok"],
-                      d["logits"], x.k, x.scale, outs=o)
+        verify_step(d["q"], d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], d["parent"], d["draft_tok"],
+                    d["logits"], x.k, x.scale, outs=o)
 
     def attn(i):
         d, o = reps[i % R], outs[i % R]
-        g.tree_attn(d["q"], d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], d["parent"], x.scale, out=o["out"])
+        tree_attn(d["q"], d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], d["parent"], x.scale, out=o["out"])
 
     def topk(i):
         d = reps[i % R]
@@ -288,8 +292,8 @@ def run_ours(args, x, cfg, rank, world, local_rank):
     hin = {k: d0[k].cpu().pin_memory() for k in ("q", "row_off", "ctx_len", "parent", "draft_tok", "logits")}
     rows = np.concatenate([np.arange(x.row_off[s] + x.ctx_len[s], x.row_off[s] + x.ctx_len[s] + x.B) for s in range(x.S)])
     rows_t = torch.from_numpy(rows).to(dev)
-    k_new = d0["k_cache"][rows_t].reshape(x.S, x.B, x.H, x.D).cpu().pin_memory()
-    v_new = d0["v_cache"][rows_t].reshape(x.S, x.B, x.H, x.D).cpu().pin_memory()
+    k_new = d0["k_cache"][rows_t].reshape(x.S, x.B, x.Hkv, x.D).cpu().pin_memory()
+    v_new = d0["v_cache"][rows_t].reshape(x.S, x.B, x.Hkv, x.D).cpu().pin_memory()
     houts = {k: v.pin_memory() for k, v in g.alloc_step_outputs(x.S, x.B, x.H, x.D, x.k, device="cpu").items()}
     h2d = sum(t.numel() * t.element_size() for t in hin.values()) + 2 * k_new.numel() * 2
     d2h = sum(t.numel() * t.element_size() for t in houts.values())
@@ -299,8 +303,8 @@ def run_ours(args, x, cfg, rank, world, local_rank):
         with torch.cuda.stream(stream):
             def host_step(i):
                 d = reps[i % R]
-                g.verify_step_host(d["k_cache"], d["v_cache"], hin["q"], k_new, v_new, hin["row_off"],
-                                   hin["ctx_len"], hin["parent"], hin["draft_tok"], hin["logits"], x.k, x.scale, houts)
+                verify_step_host(d["k_cache"], d["v_cache"], hin["q"], k_new, v_new, hin["row_off"],
+                                 hin["ctx_len"], hin["parent"], hin["draft_tok"], hin["logits"], x.k, x.scale, houts)
             for i in range(3):
                 host_step(i)
             torch.cuda.synchronize(dev)
@@ -324,7 +328,7 @@ def run_ours(args, x, cfg, rank, world, local_rank):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": cfg.name, "S": x.S, "H": x.H, "B": x.B, "D": x.D, "V": x.V, "k": x.k,
+        "config": {"workload": cfg.name, "S": x.S, "H": x.H, "Hkv": x.Hkv, "B": x.B, "D": x.D, "V": x.V, "k": x.k,
                    "ctx_len": [int(c) for c in x.ctx_len] if x.S > 1 else int(x.ctx_len[0]),
                    "l2": "rotating %d input replicas (%.2f GB total, > 2x L2)" % (R, R * footprint / 1e9),
                    "timing": "CUDA graph replay of whole steps, CUDA events, max over ranks",
@@ -356,7 +360,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--config", type=int, default=3, help="index into the workload table (0..4); default 33B")
+    ap.add_argument("--config", type=int, default=3, help="index into the workload table (0..4 the benchmark table, 5 the grouped-query workload); default 33B")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--attn-impl", choices=["mma", "umma"], default=None)

@@ -47,6 +47,7 @@ extern "C" {
 
 #define GOOSE_MAX_B     128   /* tree nodes per sequence (one 128-bit ancestor mask per node)      */
 #define GOOSE_MAX_K      16   /* top-k width                                                       */
+#define GOOSE_MAX_GROUP  16   /* query heads per key/value head (grouped-query attention)           */
 #define GOOSE_HEAD_DIM  128   /* the only supported head dimension                                 */
 #define GOOSE_MAX_V  262144   /* vocabulary size limit of goose_node_topk                          */
 #define GOOSE_STATIC_TOPK_MAX_ROWS 2048   /* row limit of goose_node_topk_static                    */
@@ -92,6 +93,17 @@ int goose_set_attn_impl(goose_ctx* ctx, int impl);
 int goose_tree_attn(goose_ctx* ctx, const void* q, const void* k_cache, const void* v_cache, int64_t kv_rows,
                     const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
                     int S, int B, int H, int D, float scale, void* out, float* lse, void* stream);
+
+/* Same for grouped-query attention, the head layout of the 8B models of the paper's evaluation (Sec. 5 set-up: 32
+ * query heads over 8 key/value heads): q and out have H heads, the caches Hkv heads, H a multiple of Hkv with
+ * H / Hkv <= GOOSE_MAX_GROUP, and query head h reads key/value head h / (H / Hkv).
+ *   k_cache, v_cache  bf16 [kv_rows][Hkv][D]
+ * Hkv == H is goose_tree_attn.  The tensor-core kernel puts the H / Hkv query heads of a group into one tile, so the
+ * key/value rows of a head are read once per group while B * (H / Hkv) <= 128, and once per
+ * ceil(B / floor(128 / (H / Hkv))) otherwise.  Other arguments, limits and errors as goose_tree_attn.          */
+int goose_tree_attn_gqa(goose_ctx* ctx, const void* q, const void* k_cache, const void* v_cache, int64_t kv_rows,
+                        const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
+                        int S, int B, int H, int Hkv, int D, float scale, void* out, float* lse, void* stream);
 
 /* Per-node argmax and top-k (Algorithm 3 step 2; App. C.1 "aggressive logit harvesting": every
  * row of the forward's logits is harvested, rejected branches included).
@@ -169,6 +181,16 @@ int goose_verify_step(goose_ctx* ctx, const void* q, void* k_cache, void* v_cach
                       int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
                       void* stream);
 
+/* The whole step for grouped-query attention: attention as goose_tree_attn_gqa (q, out with H heads), compaction
+ * over the caches' Hkv heads; everything else as goose_verify_step (which is this call with Hkv == H).       */
+int goose_verify_step_gqa(goose_ctx* ctx, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
+                          const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
+                          const int32_t* draft_tok, const void* logits, int64_t ldl,
+                          int S, int B, int H, int Hkv, int D, int V, int k, float scale,
+                          void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
+                          int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
+                          void* stream);
+
 /* Host-buffer variant of the whole step (the end-to-end call).  The prefix KV cache stays on the
  * device (k_cache / v_cache are device pointers, state carried from step to step); everything a
  * step consumes or produces is in HOST memory (pinned memory makes the copies asynchronous):
@@ -187,6 +209,17 @@ int goose_verify_step_host(goose_ctx* ctx, void* k_cache, void* v_cache, int64_t
                            void* h_out, int32_t* h_argmax, int32_t* h_topk_ids, float* h_topk_vals,
                            int32_t* h_path, int32_t* h_accept_len, int32_t* h_bonus,
                            int32_t* h_new_ctx_len, void* stream);
+
+/* Host-buffer variant of goose_verify_step_gqa: as goose_verify_step_host, with h_q / h_out of H heads and
+ * h_k_new, h_v_new bf16 [S][B][Hkv][D] (rows of the Hkv-head caches).                                        */
+int goose_verify_step_host_gqa(goose_ctx* ctx, void* k_cache, void* v_cache, int64_t kv_rows,
+                               const void* h_q, const void* h_k_new, const void* h_v_new,
+                               const int64_t* h_row_off, const int32_t* h_ctx_len,
+                               const int32_t* h_parent, const int32_t* h_draft_tok, const void* h_logits,
+                               int S, int B, int H, int Hkv, int D, int V, int k, float scale,
+                               void* h_out, int32_t* h_argmax, int32_t* h_topk_ids, float* h_topk_vals,
+                               int32_t* h_path, int32_t* h_accept_len, int32_t* h_bonus,
+                               int32_t* h_new_ctx_len, void* stream);
 
 /* ---- host routines of the loop around the verification step (all pointers below are HOST pointers) ---- */
 

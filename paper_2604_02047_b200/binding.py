@@ -21,7 +21,7 @@ EXPORTS = [
     "goose_node_topk", "goose_accept", "goose_kv_compact", "goose_verify_step",
     "goose_verify_step_host", "goose_last_status", "goose_launch_count", "goose_node_topk_static", "goose_harvest",
     "goose_build_spine_tree", "goose_pad_tree", "goose_context_match", "goose_spine_ratio_tier", "goose_spine_ema",
-    "goose_selftest_bounded_wait",
+    "goose_selftest_bounded_wait", "goose_tree_attn_gqa", "goose_verify_step_gqa", "goose_verify_step_host_gqa",
 ]
 
 ATTN_AUTO, ATTN_MMA, ATTN_UMMA = 0, 1, 2
@@ -78,6 +78,18 @@ def _dev(t: torch.Tensor, dtype: torch.dtype, name: str) -> torch.Tensor:
     return t
 
 
+def _kv_heads(k_cache: torch.Tensor, v_cache: torch.Tensor) -> int:
+    if k_cache.dim() != 3 or tuple(k_cache.shape) != tuple(v_cache.shape):
+        raise GooseError("k_cache and v_cache must both be [rows][Hkv][D]")
+    return int(k_cache.shape[1])
+
+
+def _same_heads(k_cache: torch.Tensor, v_cache: torch.Tensor, H: int, what: str) -> None:
+    if _kv_heads(k_cache, v_cache) != H:
+        raise GooseError("%s: the caches have %d heads, q has %d (grouped-query attention: use %s_gqa)"
+                         % (what, k_cache.shape[1], H, what))
+
+
 class Goose:
     """A context (workspace) on one CUDA device plus the calls of the verification step."""
 
@@ -131,6 +143,7 @@ class Goose:
         _dev(q, torch.bfloat16, "q"); _dev(k_cache, torch.bfloat16, "k_cache"); _dev(v_cache, torch.bfloat16, "v_cache")
         _dev(row_off, torch.int64, "row_off"); _dev(ctx_len, torch.int32, "ctx_len"); _dev(parent, torch.int32, "parent")
         S, B, H, D = q.shape
+        _same_heads(k_cache, v_cache, H, "tree_attn")
         if out is None:
             out = torch.empty_like(q)
         if want_lse and lse is None:
@@ -139,6 +152,24 @@ class Goose:
                                         _p(row_off), _p(ctx_len), _p(parent), ctypes.c_int(S), ctypes.c_int(B),
                                         ctypes.c_int(H), ctypes.c_int(D), ctypes.c_float(scale), _p(out), _p(lse),
                                         _stream()), "goose_tree_attn")
+        return out, lse
+
+    def tree_attn_gqa(self, q, k_cache, v_cache, row_off, ctx_len, parent, scale: float,
+                      out: Optional[torch.Tensor] = None, want_lse: bool = False,
+                      lse: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, Optional[torch.Tensor]]:
+        """Grouped-query attention: q [S][B][H][D], caches [rows][Hkv][D]; Hkv is read from the caches' shape."""
+        _dev(q, torch.bfloat16, "q"); _dev(k_cache, torch.bfloat16, "k_cache"); _dev(v_cache, torch.bfloat16, "v_cache")
+        _dev(row_off, torch.int64, "row_off"); _dev(ctx_len, torch.int32, "ctx_len"); _dev(parent, torch.int32, "parent")
+        S, B, H, D = q.shape
+        Hkv = _kv_heads(k_cache, v_cache)
+        if out is None:
+            out = torch.empty_like(q)
+        if want_lse and lse is None:
+            lse = torch.empty((S, B, H), dtype=torch.float32, device=q.device)
+        _check(self.lib.goose_tree_attn_gqa(self.h, _p(q), _p(k_cache), _p(v_cache), ctypes.c_int64(k_cache.shape[0]),
+                                            _p(row_off), _p(ctx_len), _p(parent), ctypes.c_int(S), ctypes.c_int(B),
+                                            ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D), ctypes.c_float(scale),
+                                            _p(out), _p(lse), _stream()), "goose_tree_attn_gqa")
         return out, lse
 
     def node_topk(self, logits, k: int, V: Optional[int] = None, want_vals: bool = True):
@@ -207,6 +238,7 @@ class Goose:
     def verify_step(self, q, k_cache, v_cache, row_off, ctx_len, parent, draft_tok, logits, k: int, scale: float,
                     outs: Optional[dict] = None, V: Optional[int] = None) -> dict:
         S, B, H, D = q.shape
+        _same_heads(k_cache, v_cache, H, "verify_step")
         ldl = logits.shape[1]
         V = ldl if V is None else V
         if outs is None:
@@ -220,11 +252,50 @@ class Goose:
             "goose_verify_step")
         return outs
 
+    def verify_step_gqa(self, q, k_cache, v_cache, row_off, ctx_len, parent, draft_tok, logits, k: int, scale: float,
+                        outs: Optional[dict] = None, V: Optional[int] = None) -> dict:
+        """The whole step with grouped-query attention (Hkv is read from the caches' shape)."""
+        S, B, H, D = q.shape
+        Hkv = _kv_heads(k_cache, v_cache)
+        ldl = logits.shape[1]
+        V = ldl if V is None else V
+        if outs is None:
+            outs = self.alloc_step_outputs(S, B, H, D, k, q.device)
+        _check(self.lib.goose_verify_step_gqa(
+            self.h, _p(q), _p(k_cache), _p(v_cache), ctypes.c_int64(k_cache.shape[0]), _p(row_off), _p(ctx_len),
+            _p(parent), _p(draft_tok), _p(logits), ctypes.c_int64(ldl), ctypes.c_int(S), ctypes.c_int(B),
+            ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D), ctypes.c_int(V), ctypes.c_int(k), ctypes.c_float(scale),
+            _p(outs["out"]), _p(outs.get("lse")), _p(outs["argmax"]), _p(outs["topk_ids"]), _p(outs["topk_vals"]),
+            _p(outs["path"]), _p(outs["accept_len"]), _p(outs["bonus"]), _p(outs["new_ctx_len"]), _stream()),
+            "goose_verify_step_gqa")
+        return outs
+
+    def verify_step_host_gqa(self, k_cache, v_cache, h_q, h_k_new, h_v_new, h_row_off, h_ctx_len, h_parent,
+                             h_draft_tok, h_logits, k: int, scale: float, h_outs: dict) -> dict:
+        """End-to-end call with grouped-query attention: h_k_new / h_v_new are [S][B][Hkv][D]."""
+        S, B, H, D = h_q.shape
+        Hkv = _kv_heads(k_cache, v_cache)
+        V = h_logits.shape[1]
+        for t in (h_q, h_k_new, h_v_new, h_row_off, h_ctx_len, h_parent, h_draft_tok, h_logits, *h_outs.values()):
+            if t.is_cuda or not t.is_contiguous():
+                raise GooseError("verify_step_host_gqa takes contiguous host tensors")
+        if tuple(h_k_new.shape) != (S, B, Hkv, D) or tuple(h_v_new.shape) != (S, B, Hkv, D):
+            raise GooseError("h_k_new / h_v_new must be [S][B][Hkv][D]")
+        _check(self.lib.goose_verify_step_host_gqa(
+            self.h, _p(k_cache), _p(v_cache), ctypes.c_int64(k_cache.shape[0]), _p(h_q), _p(h_k_new), _p(h_v_new),
+            _p(h_row_off), _p(h_ctx_len), _p(h_parent), _p(h_draft_tok), _p(h_logits), ctypes.c_int(S),
+            ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D), ctypes.c_int(V), ctypes.c_int(k),
+            ctypes.c_float(scale), _p(h_outs["out"]), _p(h_outs["argmax"]), _p(h_outs["topk_ids"]),
+            _p(h_outs["topk_vals"]), _p(h_outs["path"]), _p(h_outs["accept_len"]), _p(h_outs["bonus"]),
+            _p(h_outs["new_ctx_len"]), _stream()), "goose_verify_step_host_gqa")
+        return h_outs
+
     def verify_step_host(self, k_cache, v_cache, h_q, h_k_new, h_v_new, h_row_off, h_ctx_len, h_parent,
                          h_draft_tok, h_logits, k: int, scale: float, h_outs: dict) -> dict:
         """End-to-end call: per-step inputs and outputs are (pinned) host tensors; the prefix KV cache
         is device state.  Synchronises the current stream before returning."""
         S, B, H, D = h_q.shape
+        _same_heads(k_cache, v_cache, H, "verify_step_host")
         V = h_logits.shape[1]
         for t in (h_q, h_k_new, h_v_new, h_row_off, h_ctx_len, h_parent, h_draft_tok, h_logits, *h_outs.values()):
             if t.is_cuda or not t.is_contiguous():

@@ -130,8 +130,16 @@ int64_t goose_launch_count(goose_ctx* c) { return c ? c->launches : -1; }
 int goose_tree_attn(goose_ctx* c, const void* q, const void* k_cache, const void* v_cache, int64_t kv_rows,
                     const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
                     int S, int B, int H, int D, float scale, void* out, float* lse, void* stream) {
+    return goose_tree_attn_gqa(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, S, B, H, H, D, scale, out, lse,
+                               stream);
+}
+
+int goose_tree_attn_gqa(goose_ctx* c, const void* q, const void* k_cache, const void* v_cache, int64_t kv_rows,
+                        const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
+                        int S, int B, int H, int Hkv, int D, float scale, void* out, float* lse, void* stream) {
     int rc = check_shape(c, S, B, H, D);
     if (rc) return rc;
+    if (Hkv < 1 || H % Hkv != 0 || H / Hkv > GOOSE_MAX_GROUP) return GOOSE_EINVAL;
     if (!q || !k_cache || !v_cache || !row_off || !ctx_len || !parent || !out) return GOOSE_EINVAL;
     if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out)) return GOOSE_EINVAL;
     if (kv_rows < 1 || kv_rows > 0x7FFFFFFFLL) return GOOSE_EINVAL;
@@ -143,12 +151,12 @@ int goose_tree_attn(goose_ctx* c, const void* q, const void* k_cache, const void
     cudaError_t e;
     if (impl == GOOSE_ATTN_UMMA)
         e = goose::launch_tree_attn_umma(c, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_cache,
-                                         (const __nv_bfloat16*)v_cache, kv_rows, row_off, ctx_len, parent, S, B, H,
+                                         (const __nv_bfloat16*)v_cache, kv_rows, row_off, ctx_len, parent, S, B, H, Hkv,
                                          scale, (__nv_bfloat16*)out, lse, st);
     else
         e = goose::launch_tree_attn_mma(c, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_cache,
-                                        (const __nv_bfloat16*)v_cache, kv_rows, row_off, ctx_len, parent, S, B, H, scale,
-                                        (__nv_bfloat16*)out, lse, st);
+                                        (const __nv_bfloat16*)v_cache, kv_rows, row_off, ctx_len, parent, S, B, H, Hkv,
+                                        scale, (__nv_bfloat16*)out, lse, st);
     if (e != cudaSuccess) return cuda_fail(e);
     return GOOSE_OK;
 }
@@ -215,9 +223,22 @@ int goose_verify_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache,
                       void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
                       int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
                       void* stream) {
+    return goose_verify_step_gqa(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, draft_tok, logits, ldl, S, B,
+                                 H, H, D, V, k, scale, out, lse, argmax, topk_ids, topk_vals, path, accept_len, bonus,
+                                 new_ctx_len, stream);
+}
+
+int goose_verify_step_gqa(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
+                          const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
+                          const int32_t* draft_tok, const void* logits, int64_t ldl,
+                          int S, int B, int H, int Hkv, int D, int V, int k, float scale,
+                          void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
+                          int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
+                          void* stream) {
     // validate everything before enqueueing anything
     int rc = check_shape(c, S, B, H, D);
     if (rc) return rc;
+    if (Hkv < 1 || H % Hkv != 0 || H / Hkv > GOOSE_MAX_GROUP) return GOOSE_EINVAL;
     if (!q || !k_cache || !v_cache || !row_off || !ctx_len || !parent || !draft_tok || !logits || !out ||
         !argmax || !topk_ids || !path || !accept_len || !bonus || !new_ctx_len)
         return GOOSE_EINVAL;
@@ -225,13 +246,14 @@ int goose_verify_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache,
         return GOOSE_EINVAL;
     if (V < 1 || V > GOOSE_MAX_V || ldl < V || (ldl & 7) != 0 || k < 1 || k > GOOSE_MAX_K || k > V) return GOOSE_EINVAL;
     if ((long long)S * B > c->topk_rows_cap || kv_rows < 1 || kv_rows > 0x7FFFFFFFLL) return GOOSE_EINVAL;
-    rc = goose_tree_attn(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, S, B, H, D, scale, out, lse, stream);
+    rc = goose_tree_attn_gqa(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, S, B, H, Hkv, D, scale, out, lse,
+                             stream);
     if (rc) return rc;
     rc = goose_node_topk(c, logits, S * B, V, ldl, k, argmax, topk_ids, topk_vals, stream);
     if (rc) return rc;
     // acceptance walk + compaction in one launch (same results as goose_accept followed by goose_kv_compact)
     cudaError_t e = goose::launch_accept_compact(c, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, row_off, ctx_len,
-                                                 draft_tok, parent, argmax, S, B, H, kv_rows, path, accept_len, bonus,
+                                                 draft_tok, parent, argmax, S, B, Hkv, kv_rows, path, accept_len, bonus,
                                                  new_ctx_len, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(e);
     return GOOSE_OK;
@@ -245,8 +267,22 @@ int goose_verify_step_host(goose_ctx* c, void* k_cache, void* v_cache, int64_t k
                            void* h_out, int32_t* h_argmax, int32_t* h_topk_ids, float* h_topk_vals,
                            int32_t* h_path, int32_t* h_accept_len, int32_t* h_bonus,
                            int32_t* h_new_ctx_len, void* stream) {
+    return goose_verify_step_host_gqa(c, k_cache, v_cache, kv_rows, h_q, h_k_new, h_v_new, h_row_off, h_ctx_len, h_parent,
+                                      h_draft_tok, h_logits, S, B, H, H, D, V, k, scale, h_out, h_argmax, h_topk_ids,
+                                      h_topk_vals, h_path, h_accept_len, h_bonus, h_new_ctx_len, stream);
+}
+
+int goose_verify_step_host_gqa(goose_ctx* c, void* k_cache, void* v_cache, int64_t kv_rows,
+                               const void* h_q, const void* h_k_new, const void* h_v_new,
+                               const int64_t* h_row_off, const int32_t* h_ctx_len,
+                               const int32_t* h_parent, const int32_t* h_draft_tok, const void* h_logits,
+                               int S, int B, int H, int Hkv, int D, int V, int k, float scale,
+                               void* h_out, int32_t* h_argmax, int32_t* h_topk_ids, float* h_topk_vals,
+                               int32_t* h_path, int32_t* h_accept_len, int32_t* h_bonus,
+                               int32_t* h_new_ctx_len, void* stream) {
     int rc = check_shape(c, S, B, H, D);
     if (rc) return rc;
+    if (Hkv < 1 || H % Hkv != 0 || H / Hkv > GOOSE_MAX_GROUP) return GOOSE_EINVAL;
     if (!k_cache || !v_cache || !h_q || !h_k_new || !h_v_new || !h_row_off || !h_ctx_len || !h_parent ||
         !h_draft_tok || !h_logits || !h_out || !h_argmax || !h_topk_ids || !h_path || !h_accept_len || !h_bonus ||
         !h_new_ctx_len)
@@ -284,7 +320,7 @@ int goose_verify_step_host(goose_ctx* c, void* k_cache, void* v_cache, int64_t k
         c->stage_bytes = off;
     }
     char* d = static_cast<char*>(c->stage);
-    const size_t row_bytes = (size_t)H * D * 2;
+    const size_t row_bytes = (size_t)Hkv * D * 2;       // one cache row
     GOOSE_CUDA(cudaMemcpyAsync(d + o_q, h_q, n_q, cudaMemcpyHostToDevice, st));
     for (int s = 0; s < S; ++s) {
         size_t dst = (size_t)(h_row_off[s] + h_ctx_len[s]) * row_bytes;
@@ -298,11 +334,11 @@ int goose_verify_step_host(goose_ctx* c, void* k_cache, void* v_cache, int64_t k
     GOOSE_CUDA(cudaMemcpyAsync(d + o_ctx, h_ctx_len, S * 4, cudaMemcpyHostToDevice, st));
     GOOSE_CUDA(cudaMemcpyAsync(d + o_parent, h_parent, rows * 4, cudaMemcpyHostToDevice, st));
     GOOSE_CUDA(cudaMemcpyAsync(d + o_tok, h_draft_tok, rows * 4, cudaMemcpyHostToDevice, st));
-    rc = goose_verify_step(c, d + o_q, k_cache, v_cache, kv_rows, (const int64_t*)(d + o_rowoff),
-                           (const int32_t*)(d + o_ctx), (const int32_t*)(d + o_parent), (const int32_t*)(d + o_tok),
-                           d + o_logits, V, S, B, H, D, V, k, scale, d + o_out, nullptr, (int32_t*)(d + o_argmax),
-                           (int32_t*)(d + o_ids), (float*)(d + o_vals), (int32_t*)(d + o_path),
-                           (int32_t*)(d + o_alen), (int32_t*)(d + o_bonus), (int32_t*)(d + o_newctx), stream);
+    rc = goose_verify_step_gqa(c, d + o_q, k_cache, v_cache, kv_rows, (const int64_t*)(d + o_rowoff),
+                               (const int32_t*)(d + o_ctx), (const int32_t*)(d + o_parent), (const int32_t*)(d + o_tok),
+                               d + o_logits, V, S, B, H, Hkv, D, V, k, scale, d + o_out, nullptr, (int32_t*)(d + o_argmax),
+                               (int32_t*)(d + o_ids), (float*)(d + o_vals), (int32_t*)(d + o_path),
+                               (int32_t*)(d + o_alen), (int32_t*)(d + o_bonus), (int32_t*)(d + o_newctx), stream);
     if (rc) return rc;
     GOOSE_CUDA(cudaMemcpyAsync(h_out, d + o_out, n_q, cudaMemcpyDeviceToHost, st));
     GOOSE_CUDA(cudaMemcpyAsync(h_argmax, d + o_argmax, rows * 4, cudaMemcpyDeviceToHost, st));

@@ -87,7 +87,7 @@ __global__ void __launch_bounds__(256)
 tree_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ kc,
                      const __nv_bfloat16* __restrict__ vc, const int64_t* __restrict__ row_off,
                      const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ parent,
-                     int B, int H, int64_t kv_rows, float scale_log2, int splits,
+                     int B, int H, int Hkv, int64_t kv_rows, float scale_log2, int splits,
                      float* __restrict__ partials, int32_t* __restrict__ head_counters,
                      int32_t* __restrict__ status, __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -96,6 +96,9 @@ tree_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     const int split = blockIdx.x, h = blockIdx.y, s = blockIdx.z;
     const int tid = threadIdx.x, nthreads = blockDim.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, t4 = lane & 3;
+    // grouped-query attention: query head h reads key/value head h / (H / Hkv); every query head streams its
+    // key/value head by itself here (the tcgen05 kernel shares the stream across the group)
+    const int hk = h / (H / Hkv);
     pdl_wait();
     pdl_trigger();
     const int ctx = max(ctx_len[s], 0);                    // device data: a negative length is treated as 0
@@ -141,13 +144,13 @@ tree_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
 
     // ---- stream the tiles
     if (t_begin < t_end && !bad) {
-        load_tile_async(smem, kc, vc, row0, t_begin * kKT, n_keys, H, h, tid, nthreads);
+        load_tile_async(smem, kc, vc, row0, t_begin * kKT, n_keys, Hkv, hk, tid, nthreads);
     }
     cp_async_commit();
     for (int t = t_begin; t < t_end && !bad; ++t) {
         const int stage = (t - t_begin) & 1;
         if (t + 1 < t_end)
-            load_tile_async(smem + (stage ^ 1) * 2 * kTileBytes, kc, vc, row0, (t + 1) * kKT, n_keys, H, h, tid, nthreads);
+            load_tile_async(smem + (stage ^ 1) * 2 * kTileBytes, kc, vc, row0, (t + 1) * kKT, n_keys, Hkv, hk, tid, nthreads);
         cp_async_commit();
         cp_async_wait<1>();
         __syncthreads();
@@ -319,7 +322,7 @@ int mma_splits(const goose_ctx* c, int S, int H) {
 
 cudaError_t launch_tree_attn_mma(goose_ctx* c, const __nv_bfloat16* q, const __nv_bfloat16* kc,
                                  const __nv_bfloat16* vc, int64_t kv_rows, const int64_t* row_off, const int32_t* ctx_len,
-                                 const int32_t* parent, int S, int B, int H, float scale,
+                                 const int32_t* parent, int S, int B, int H, int Hkv, float scale,
                                  __nv_bfloat16* out, float* lse, cudaStream_t st) {
     if (S == 0 || H == 0) return cudaSuccess;
     int splits = mma_splits(c, S, H);
@@ -327,7 +330,7 @@ cudaError_t launch_tree_attn_mma(goose_ctx* c, const __nv_bfloat16* q, const __n
     if (warps < 4) warps = 4;
     dim3 grid(splits, H, S);
     cudaError_t e = launch_pdl(tree_attn_mma_kernel, grid, dim3(warps * 32), kMmaSmem, st, q, kc, vc, row_off, ctx_len,
-                               parent, B, H, kv_rows, scale * kLog2e, splits, c->partials, c->head_counters, c->status, out, lse);
+                               parent, B, H, Hkv, kv_rows, scale * kLog2e, splits, c->partials, c->head_counters, c->status, out, lse);
     c->launches++;
     return e;
 }

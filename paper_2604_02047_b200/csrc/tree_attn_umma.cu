@@ -16,7 +16,10 @@
 //                                  shared memory in the canonical 128-byte-swizzled K-major layout,
 //                                  lazy rescaling of O in TMEM, epilogue (output or partial).
 // All B <= 128 query rows ride in one M = 128 MMA; rows >= B compute on don't-care data and are
-// never written out.  The tree part of the mask (Sec. 4 Stage 1: a node attends to the prefix and to
+// never written out.  Grouped-query attention (H query heads over Hkv key/value heads, g = H / Hkv) stacks the g
+// query heads of a group into the same M tile -- row r = (node r / g, group member r % g) -- so a K/V tile is
+// streamed once per group; when B * g > 128 the nodes are cut into M tiles of floor(128 / g) nodes and the K/V of a
+// head is streamed once per M tile.  A "head" of the work list below is one (M tile, key/value head) pair.  The tree part of the mask (Sec. 4 Stage 1: a node attends to the prefix and to
 // its root-to-node ancestors) is a per-row 128-bit ancestor set built from parent[].
 //
 // Every wait in this file is bounded: when a wait runs out of polls the CTA raises an abort flag,
@@ -130,10 +133,10 @@ __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, unsigned long long* bar,
-                                            int c0, int c1, int c2) {
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, unsigned long long* bar,
+                                            int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
 __device__ __forceinline__ void tma_load_3d_hint(void* dst, const CUtensorMap* map, unsigned long long* bar,
                                                  int c0, int c1, int c2, unsigned long long policy) {
@@ -222,7 +225,7 @@ __device__ __forceinline__ bool group_sync(Header* hd, uint32_t& n, int32_t* sta
 // ---------------------------------------------------------------- work partition (same code in every role)
 struct Work {
     const int32_t* ctx_len;
-    int S, H, B, G;
+    int S, H, B, G;           // H = heads of the work list = M tiles x key/value heads (M-tile-major)
     long long total;          // all items
     bool small;               // total * (G + 1) fits 31 bits: 32-bit arithmetic (64-bit division is slow on the GPU)
     // ctx_len comes from device memory: a negative value is treated as 0 (the tree rows alone)
@@ -273,13 +276,18 @@ struct Cursor {               // walks items in order
 };
 
 // ---------------------------------------------------------------- the kernel
+// kGrouped = false is multi-head attention: one query head per key/value head and one M tile per sequence are
+// compile-time facts there (the per-row index arithmetic folds away); kGrouped = true takes them from the arguments.
+template <bool kGrouped>
 __global__ void __launch_bounds__(kThreads, 1)
 tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                       const __grid_constant__ CUtensorMap tmap_v, const int64_t* __restrict__ row_off,
                       const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ parent,
-                      int S, int B, int H, int64_t kv_rows, float scale_log2, float* __restrict__ partials,
+                      int S, int B, int H, int Hkv_arg, int g_arg, int nb_arg, int64_t kv_rows, float scale_log2,
+                      float* __restrict__ partials,
                       int32_t* __restrict__ status,
                       __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+    const int Hkv = kGrouped ? Hkv_arg : H, g = kGrouped ? g_arg : 1, nb = kGrouped ? nb_arg : B;
     extern __shared__ unsigned char smem_raw[];
     Header* hd = reinterpret_cast<Header*>(smem_raw);
     unsigned char* buf = reinterpret_cast<unsigned char*>(
@@ -320,7 +328,9 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     pdl_wait();
     pdl_trigger();
     Work wk;
-    wk.ctx_len = ctx_len; wk.S = S; wk.H = H; wk.B = B; wk.G = gridDim.x;
+    // g query heads per key/value head, nb nodes per M tile (nb * g <= 128), n_mt M tiles per sequence
+    const int n_mt = kGrouped ? (B + nb - 1) / nb : 1;
+    wk.ctx_len = ctx_len; wk.S = S; wk.H = n_mt * Hkv; wk.B = B; wk.G = gridDim.x;
     wk.init();
     const long long w_begin = wk.cta_start(blockIdx.x), w_end = wk.cta_start(blockIdx.x + 1);
 
@@ -344,9 +354,12 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                     const uint32_t qb = seg & 1;           // seg = index of this segment
                     ok = mbar_wait(hd, &hd->q_empty[qb], ((seg >> 1) & 1) ^ 1, status);
                     if (!ok) break;
-                    mbar_expect_tx(&hd->q_full[qb], (uint32_t)B * 256u);
-                    tma_load_3d(q_smem + qb * kQBytes, &tmap_q, &hd->q_full[qb], 0, cu.h, cu.s * B);
-                    tma_load_3d(q_smem + qb * kQBytes + kHalfBytes, &tmap_q, &hd->q_full[qb], 64, cu.h, cu.s * B);
+                    // box = nb nodes x g heads x 64 dims: lands as rows r = node * g + member (rows past the
+                    // sequence's last node hold the next sequence's queries or the zero fill: never written out)
+                    const int mt = kGrouped ? cu.h / Hkv : 0, hk = cu.h - mt * Hkv;
+                    mbar_expect_tx(&hd->q_full[qb], (uint32_t)(nb * g) * 256u);
+                    tma_load_4d(q_smem + qb * kQBytes, &tmap_q, &hd->q_full[qb], 0, 0, hk, cu.s * B + mt * nb);
+                    tma_load_4d(q_smem + qb * kQBytes + kHalfBytes, &tmap_q, &hd->q_full[qb], 64, 0, hk, cu.s * B + mt * nb);
                     ++seg;                                 // segments whose Q load has been issued
                     const int s0 = cu.s, h0 = cu.h;
                     while (ok && cu.w < w_end && cu.s == s0 && cu.h == h0) {
@@ -358,8 +371,8 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                             unsigned char* dst = kv_smem + st * kStageBytes;
                             mbar_expect_tx(&hd->kv_full[st], kStageBytes);
                             const CUtensorMap* mp = kv ? &tmap_v : &tmap_k;
-                            tma_load_3d_hint(dst, mp, &hd->kv_full[st], 0, cu.h, krow, pol_stream);
-                            tma_load_3d_hint(dst + kHalfBytes, mp, &hd->kv_full[st], 64, cu.h, krow, pol_stream);
+                            tma_load_3d_hint(dst, mp, &hd->kv_full[st], 0, hk, krow, pol_stream);
+                            tma_load_3d_hint(dst + kHalfBytes, mp, &hd->kv_full[st], 64, hk, krow, pol_stream);
                             ++ring;
                             TRACE(0, tn, 2);
                         }
@@ -442,13 +455,14 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
             // =========================================================== softmax / epilogue (128 threads)
             const int row = 32 * (warp & 3) + lane;        // TMEM lane == query row
             const uint32_t lane_sel = (uint32_t)(32 * (warp & 3)) << 16;
-            const bool warp_has_rows = 32 * (warp & 3) < B;
+            const int i_local = kGrouped ? row / g : row;  // row = (node of the M tile, head of the group)
+            const int member = row - i_local * g;
             const int sm_tid = threadIdx.x - 64;           // 0..127
             Cursor cu; cu.seek(wk, w_begin);
             uint32_t jg = 0, seg = 0, gsync = 0;
             bool ok = true;
             uint32_t v[128];
-            int cur_s = -1;
+            int cur_s = -1, cur_mt = -1;
             bool bad = false;
             uint32_t anc[4] = {0, 0, 0, 0};
             TRACE_DECL;
@@ -456,15 +470,20 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
 
             while (ok && cu.w < w_end) {
                 const int s0 = cu.s, h0 = cu.h, T = cu.T;
+                const int mt = kGrouped ? h0 / Hkv : 0, hk = h0 - mt * Hkv;
+                const int node = mt * nb + i_local;        // tree node of this thread's row
+                const bool row_valid = i_local < nb && node < B;
+                const bool warp_has_rows = 32 * (warp & 3) < min(nb, B - mt * nb) * g;
                 const int ctx = max(ctx_len[s0], 0);
                 const int n_keys = ctx + B;
                 const int32_t* par = parent + (size_t)s0 * B;
                 const int t_first = cu.t;
                 // new sequence: validate parent[] (all 128 threads reach the same verdict) and rebuild
                 // this row's ancestor set; consecutive segments of one sequence reuse both
-                if (s0 != cur_s) {
+                const bool new_seq = s0 != cur_s;
+                if (new_seq) {
                     cur_s = s0;
-                    if (row < B) {
+                    if (row < B) {                         // thread r stages parent[r] (independent of the row stacking)
                         int p = par[row];
                         hd->par[row] = p;
                         if ((row == 0) ? (p != -1) : (p < 0 || p >= row)) hd->bad_parent = 1;
@@ -479,12 +498,18 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                     ok = ok && group_sync(hd, gsync, status);
                     if (!ok) break;
                     if (sm_tid == 0 && bad) { hd->bad_parent = 0; if (!bad_rows) atomicOr(&status[s0], GOOSE_ST_BAD_PARENT); }
+                }
+                if (new_seq || mt != cur_mt) {             // hd->par[] still holds this sequence's parents
+                    cur_mt = mt;
                     anc[0] = anc[1] = anc[2] = anc[3] = 0;
-                    if (row < B) {
+                    if (row_valid) {
                         if (bad) {
-                            anc[row >> 5] = 1u << (row & 31);
+                            const uint32_t bit = 1u << (node & 31);
+                            const int wsel = node >> 5;
+                            anc[0] = (wsel == 0) ? bit : 0; anc[1] = (wsel == 1) ? bit : 0;
+                            anc[2] = (wsel == 2) ? bit : 0; anc[3] = (wsel == 3) ? bit : 0;
                         } else {
-                            int vtx = row;
+                            int vtx = node;
                             for (int step = 0; step < B && vtx >= 0; ++step) {
                                 uint32_t bit = 1u << (vtx & 31);
                                 int wsel = vtx >> 5;
@@ -630,10 +655,11 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 tc_fence_before();
                 mbar_arrive(&hd->o_free);                  // TMEM O may be overwritten by the next segment
 
+                const int hq = hk * g + member;            // query head of this row
                 if (whole_head) {
-                    if (row < B) {
+                    if (row_valid) {
                         const float inv = bad ? 0.f : 1.f / l_run;
-                        uint4* dst = reinterpret_cast<uint4*>(out + (((size_t)s0 * B + row) * H + h0) * kHeadDim);
+                        uint4* dst = reinterpret_cast<uint4*>(out + (((size_t)s0 * B + node) * H + hq) * kHeadDim);
 #pragma unroll
                         for (int ch = 0; ch < 16; ++ch) {
                             uint32_t pk[4];
@@ -643,14 +669,14 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                                                                __uint_as_float(v[ch * 8 + 2 * e + 1]) * inv);
                             dst[ch] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         }
-                        if (lse) lse[((size_t)s0 * B + row) * H + h0] = bad ? 0.f : (m_run + log2f(l_run)) * kLn2;
+                        if (lse) lse[((size_t)s0 * B + node) * H + hq] = bad ? 0.f : (m_run + log2f(l_run)) * kLn2;
                     }
                 } else {
                     // partial -> workspace slot of this CTA (combined by tree_attn_combine_kernel): O/l in fp16
                     // (relative error 2^-11, far below the bf16 rounding of the final output), m and l in fp32
                     const int slot = 2 * blockIdx.x + (t_first == 0 ? 1 : 0);
                     float* part = partials + (size_t)slot * kUmmaPartFloats;
-                    if (row < B) {
+                    if (row_valid) {
                         // invalid parent[]: a neutral partial (O = 0; the head's first part carries weight 1)
                         // makes the combine kernel produce the defined zero output without re-validating
                         const float inv = (bad || l_run == 0.f) ? 0.f : 1.f / l_run;
@@ -688,29 +714,36 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
 }
 
 // ---------------------------------------------------------------- combine of the split-KV partials
-// Grid (row groups of 32, H, S), 256 threads.  A head that one CTA of the main kernel covered entirely
-// was written directly and is skipped; any other head is the merge of its CTAs' partials:
+// Grid (row groups of 32, M tiles x key/value heads, S), 256 threads.  A head of the work list that one CTA of the
+// main kernel covered entirely was written directly and is skipped; any other is the merge of its CTAs' partials:
 //   M = max m_p,  L = sum l_p 2^(m_p - M),  out = sum_p 2^(m_p - M) O_p / L.
 // Lane <-> row (coalesced float4 loads of the transposed partial layout), warp <-> 16 output columns.
+template <bool kGrouped>
 __global__ void __launch_bounds__(kCombineThreads)
-tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, int S, int B, int H, int G,
+tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, int S, int B, int H, int Hkv_arg, int g_arg, int nb_arg, int G,
                          const float* __restrict__ partials, __nv_bfloat16* __restrict__ out,
                          float* __restrict__ lse) {
-    const int rg = blockIdx.x, h = blockIdx.y, s = blockIdx.z;
+    const int Hkv = kGrouped ? Hkv_arg : H, g = kGrouped ? g_arg : 1, nb = kGrouped ? nb_arg : B;
+    const int rg = blockIdx.x, h = blockIdx.y, s = blockIdx.z;   // h = head of the work list (M tile, KV head)
+    const int Hw = gridDim.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // The partition arithmetic needs only ctx_len[], which is final before this kernel's CTAs can start: the main
     // kernel triggers its dependents after its own pdl_wait(), i.e. after whatever produced ctx_len[] completed.
     // So all of it runs before the wait, and the partial loads are issued the moment the main grid is done.
     Work wk;
-    wk.ctx_len = ctx_len; wk.S = S; wk.H = H; wk.B = B; wk.G = G;
+    wk.ctx_len = ctx_len; wk.S = S; wk.H = Hw; wk.B = B; wk.G = G;
     wk.init();
     long long off = 0;
-    for (int ss = 0; ss < s; ++ss) off += (long long)H * wk.tiles(ss);
+    for (int ss = 0; ss < s; ++ss) off += (long long)Hw * wk.tiles(ss);
     const int T = wk.tiles(s);
     const long long head_first = off + (long long)h * T;
     const int c_lo = wk.cta_of(head_first), c_hi = wk.cta_of(head_first + T - 1);
     const bool whole = c_lo == c_hi;                       // written directly by the main kernel
-    const int row = rg * 32 + lane;
+    const int row = rg * 32 + lane;                        // row of the M tile = (node of the tile, head of the group)
+    const int mt = kGrouped ? h / Hkv : 0, hk = h - mt * Hkv;
+    const int i_local = kGrouped ? row / g : row, node = mt * nb + i_local;
+    const int hq = hk * g + (row - i_local * g);
+    const bool row_valid = i_local < nb && node < B;
     // CTA c's partial for this head sits in slot 2c, or 2c+1 when its segment starts at the head's first tile,
     // which only the first CTA can do.  With fewer items than CTAs some CTAs in [c_lo, c_hi] are empty.
     const int flag_lo = wk.cta_start(c_lo) <= head_first ? 1 : 0;
@@ -719,7 +752,7 @@ tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, int S, int B, int 
     // complete" implying "the main grid is complete"
     pdl_wait();                                            // the main kernel's partials are complete and visible
     pdl_trigger();
-    if (whole || row >= B) return;
+    if (whole || !row_valid) return;
     float M_run = -INFINITY, L_run = 0.f;
     float acc[16];                                         // warp w owns columns 16w .. 16w+15 (column groups 2w, 2w+1)
 #pragma unroll
@@ -769,17 +802,31 @@ tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, int S, int B, int 
         M_run = M_new;
     }
     const float inv = 1.f / L_run;
-    uint4* dst = reinterpret_cast<uint4*>(out + (((size_t)s * B + row) * H + h) * kHeadDim + 16 * warp);
+    uint4* dst = reinterpret_cast<uint4*>(out + (((size_t)s * B + node) * H + hq) * kHeadDim + 16 * warp);
 #pragma unroll
     for (int u = 0; u < 2; ++u)
         dst[u] = make_uint4(pack_bf16x2(acc[8 * u] * inv, acc[8 * u + 1] * inv), pack_bf16x2(acc[8 * u + 2] * inv, acc[8 * u + 3] * inv),
                             pack_bf16x2(acc[8 * u + 4] * inv, acc[8 * u + 5] * inv), pack_bf16x2(acc[8 * u + 6] * inv, acc[8 * u + 7] * inv));
-    if (lse && warp == 0) lse[((size_t)s * B + row) * H + h] = (M_run + log2f(L_run)) * kLn2;
+    if (lse && warp == 0) lse[((size_t)s * B + node) * H + hq] = (M_run + log2f(L_run)) * kLn2;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// bf16 queries [rows][Hkv][g][128] -> 4-D map, box = 64 x g x 1 x box_rows: the g query heads of one key/value
+// head for box_rows consecutive nodes, landing as rows (node, member) of one 128-byte-swizzled tile
+bool make_q_map(void* fn, CUtensorMap* map, const void* base, int64_t rows, int Hkv, int g, int box_rows) {
+    cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)g, (cuuint64_t)Hkv, (cuuint64_t)rows};
+    cuuint64_t strides[3] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)g * kHeadDim * 2, (cuuint64_t)Hkv * g * kHeadDim * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)g, 1, (cuuint32_t)box_rows};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = reinterpret_cast<EncodeTiledFn>(fn)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base),
+                                                     dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
 
 // bf16 tensor [rows][H][128] -> 3-D map, box = 64 x 1 x box_rows, 128-byte swizzle, zero fill out of bounds
 bool make_map(void* fn, CUtensorMap* map, const void* base, int64_t rows, int H, int box_rows) {
@@ -830,7 +877,9 @@ cudaError_t launch_bounded_wait_selftest(goose_ctx* c, long long limit_cycles, i
 }
 
 cudaError_t init_umma_kernel() {
-    return cudaFuncSetAttribute(tree_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmem);
+    cudaError_t e = cudaFuncSetAttribute(tree_attn_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(tree_attn_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmem);
 }
 
 int auto_attn_impl(const goose_ctx* c, int S, int B, int H) {
@@ -843,27 +892,33 @@ int auto_attn_impl(const goose_ctx* c, int S, int B, int H) {
 
 cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __nv_bfloat16* kc,
                                   const __nv_bfloat16* vc, int64_t kv_rows, const int64_t* row_off,
-                                  const int32_t* ctx_len, const int32_t* parent, int S, int B, int H,
+                                  const int32_t* ctx_len, const int32_t* parent, int S, int B, int H, int Hkv,
                                   float scale, __nv_bfloat16* out, float* lse, cudaStream_t st) {
     if (!c->encode_tiled) return cudaErrorNotSupported;
     if (S == 0) return cudaSuccess;
+    const int g = H / Hkv;                              // query heads per key/value head (validated by the caller)
+    const int nb = B * g <= kTile ? B : kTile / g;      // nodes per M tile
+    const int n_mt = (B + nb - 1) / nb;
     CUtensorMap mq, mk, mv;
-    if (!make_map(c->encode_tiled, &mq, q, (int64_t)S * B, H, B) ||
-        !make_map(c->encode_tiled, &mk, kc, kv_rows, H, kTile) ||
-        !make_map(c->encode_tiled, &mv, vc, kv_rows, H, kTile))
+    if (!make_q_map(c->encode_tiled, &mq, q, (int64_t)S * B, Hkv, g, nb) ||
+        !make_map(c->encode_tiled, &mk, kc, kv_rows, Hkv, kTile) ||
+        !make_map(c->encode_tiled, &mv, vc, kv_rows, Hkv, kTile))
         return cudaErrorInvalidValue;
     int grid = c->num_sms;
     if (2 * grid > c->n_slots) grid = c->n_slots / 2;
-    cudaError_t e = launch_pdl(tree_attn_umma_kernel, dim3(grid), dim3(kThreads), kUmmaSmem, st, mq, mk, mv, row_off,
-                               ctx_len, parent, S, B, H, kv_rows, scale * kLog2e, c->partials, c->status, out, lse);
+    const bool grouped = g > 1;
+    cudaError_t e = launch_pdl(grouped ? tree_attn_umma_kernel<true> : tree_attn_umma_kernel<false>, dim3(grid),
+                               dim3(kThreads), kUmmaSmem, st, mq, mk, mv, row_off, ctx_len, parent, S, B, H, Hkv, g, nb,
+                               kv_rows, scale * kLog2e, c->partials, c->status, out, lse);
     c->launches++;
     if (e != cudaSuccess) return e;
 #ifdef GOOSE_TRACE
     if (getenv("GOOSE_SKIP_COMBINE")) return e;       // debug build only: time the main kernel alone
 #endif
-    dim3 cgrid((B + 31) / 32, H, S);
+    dim3 cgrid((nb * g + 31) / 32, n_mt * Hkv, S);
     const float* parts = c->partials;
-    e = launch_pdl(tree_attn_combine_kernel, cgrid, dim3(kCombineThreads), 0, st, ctx_len, S, B, H, grid, parts, out, lse);
+    e = launch_pdl(grouped ? tree_attn_combine_kernel<true> : tree_attn_combine_kernel<false>, cgrid,
+                   dim3(kCombineThreads), 0, st, ctx_len, S, B, H, Hkv, g, nb, grid, parts, out, lse);
     c->launches++;
     return e;
 }

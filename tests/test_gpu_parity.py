@@ -43,8 +43,9 @@ def _run_attn(goose, x, impl, want_lse=True):
     goose.set_attn_impl(impl)
     try:
         d = binding.to_device(x)
-        out, lse = goose.tree_attn(d["q"], d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], d["parent"],
-                                   x.scale, want_lse=want_lse)
+        call = goose.tree_attn if x.Hkv == x.H else goose.tree_attn_gqa
+        out, lse = call(d["q"], d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], d["parent"],
+                        x.scale, want_lse=want_lse)
         torch.cuda.synchronize()
         st = goose.last_status(x.S)
     finally:
@@ -315,14 +316,16 @@ def _check_step(goose, oracle, x, n_rows=192, host=False):
         hin = {k_: v.cpu().pin_memory() for k_, v in d.items()}
         rows = np.concatenate([np.arange(x.row_off[s] + x.ctx_len[s], x.row_off[s] + x.ctx_len[s] + x.B) for s in range(x.S)])
         rows_t = torch.from_numpy(rows).cuda()
-        k_new = d["k_cache"][rows_t].reshape(x.S, x.B, x.H, x.D).cpu().pin_memory()
-        v_new = d["v_cache"][rows_t].reshape(x.S, x.B, x.H, x.D).cpu().pin_memory()
+        k_new = d["k_cache"][rows_t].reshape(x.S, x.B, x.Hkv, x.D).cpu().pin_memory()
+        v_new = d["v_cache"][rows_t].reshape(x.S, x.B, x.Hkv, x.D).cpu().pin_memory()
         d["k_cache"][rows_t] = 0; d["v_cache"][rows_t] = 0     # the call must put the tree rows in place itself
-        o = goose.verify_step_host(d["k_cache"], d["v_cache"], hin["q"], k_new, v_new, hin["row_off"], hin["ctx_len"],
-                                   hin["parent"], hin["draft_tok"], hin["logits"], x.k, x.scale, houts)
+        call = goose.verify_step_host if x.Hkv == x.H else goose.verify_step_host_gqa
+        o = call(d["k_cache"], d["v_cache"], hin["q"], k_new, v_new, hin["row_off"], hin["ctx_len"],
+                 hin["parent"], hin["draft_tok"], hin["logits"], x.k, x.scale, houts)
     else:
-        o = goose.verify_step(d["q"], d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], d["parent"],
-                              d["draft_tok"], d["logits"], x.k, x.scale)
+        call = goose.verify_step if x.Hkv == x.H else goose.verify_step_gqa
+        o = call(d["q"], d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], d["parent"],
+                 d["draft_tok"], d["logits"], x.k, x.scale)
         torch.cuda.synchronize()
     assert not goose.last_status(x.S).any()
     ram, rids, rvals = oracle.node_topk(x.logits, x.k)

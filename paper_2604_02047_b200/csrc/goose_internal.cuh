@@ -101,9 +101,11 @@ int mma_splits(const goose_ctx* c, int S, int H);
 // per-device kernel attributes (dynamic shared memory limits); called once from goose_create
 cudaError_t init_mma_kernel();
 cudaError_t init_umma_kernel();
+cudaError_t init_topk_kernel();
 inline cudaError_t init_kernels(goose_ctx*) {
     cudaError_t e = init_mma_kernel();
-    return e != cudaSuccess ? e : init_umma_kernel();
+    if (e == cudaSuccess) e = init_umma_kernel();
+    return e != cudaSuccess ? e : init_topk_kernel();
 }
 
 // kernel choice of GOOSE_ATTN_AUTO

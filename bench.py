@@ -34,7 +34,8 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM traffic per attention launch from the ncu capture summarised under profiles/ (bytes), per config
 # name; None = not captured for that workload.
 NCU_TRAFFIC_BYTES = {"33b": 227_470_000,    # tree_attn_umma_kernel: 223.29 MB read + 4.2 MB written per launch
-                     "13b": 89_450_000}     # 86.42 MB read + 3.0 MB written
+                     "13b": 89_450_000,
+                     "gqa8b": 169_570_000}  # 165.0 MB read + 3.2-5.8 MB written per launch (two launches averaged)     # 86.42 MB read + 3.0 MB written
 
 
 def _peaks():
@@ -237,14 +238,16 @@ def run_ours(args, x, cfg, rank, world, local_rank):
             step(i)
         stream.synchronize()
         # one CUDA graph per leg: a full rotation over the replicas
-        def capture(fn):
+        def capture(fn, n=R):
             gr = torch.cuda.CUDAGraph()
             n0 = g.launch_count()
             with torch.cuda.graph(gr, stream=stream, capture_error_mode="thread_local"):
-                for i in range(R):
+                for i in range(n):
                     fn(i)
-            return gr, (g.launch_count() - n0) // R
+            return gr, (g.launch_count() - n0) // n
         g_step, launches_per_step = capture(step)
+        # K steps = whole rotations plus one partial rotation, which gets a graph of its own
+        g_tail = capture(step, args.steps % R)[0] if args.steps % R else None
         g_attn, _ = capture(attn)
         g_topk, _ = capture(topk)
         g_harv, _ = capture(harvest)
@@ -267,11 +270,10 @@ def run_ours(args, x, cfg, rank, world, local_rank):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
             done = 0
-            while done < args.steps:                      # exactly K steps: whole rotations, then a partial one
-                if args.steps - done >= R:
-                    g_step.replay(); done += R
-                else:
-                    step(done); done += 1
+            while args.steps - done >= R:                 # exactly K steps: whole rotations, then the partial one
+                g_step.replay(); done += R
+            if g_tail is not None:
+                g_tail.replay(); done += args.steps % R
             e1.record(stream)
             torch.cuda.synchronize(dev)
             dist_barrier()

@@ -249,8 +249,13 @@ int goose_verify_step_gqa(goose_ctx* c, const void* q, void* k_cache, void* v_ca
     rc = goose_tree_attn_gqa(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, S, B, H, Hkv, D, scale, out, lse,
                              stream);
     if (rc) return rc;
-    rc = goose_node_topk(c, logits, S * B, V, ldl, k, argmax, topk_ids, topk_vals, stream);
-    if (rc) return rc;
+    // the logits are an input of the step: complete before the attention kernels above started, which do not touch
+    // them -- so the top-k kernel may read them while the attention merge is still running
+    if (S > 0) {
+        cudaError_t et = goose::launch_node_topk(c, (const __nv_bfloat16*)logits, S * B, V, ldl, k, argmax, topk_ids, topk_vals,
+                                                 nullptr, static_cast<cudaStream_t>(stream), /*inputs_ready=*/true);
+        if (et != cudaSuccess) return cuda_fail(et);
+    }
     // acceptance walk + compaction in one launch (same results as goose_accept followed by goose_kv_compact)
     cudaError_t e = goose::launch_accept_compact(c, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, row_off, ctx_len,
                                                  draft_tok, parent, argmax, S, B, Hkv, kv_rows, path, accept_len, bonus,

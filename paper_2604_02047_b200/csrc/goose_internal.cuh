@@ -70,8 +70,10 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 #endif
 
 // launchers (each returns a cudaError_t from the launch)
+// inputs_ready: the logits were complete before the kernel preceding this one in the stream started (see the kernel)
 cudaError_t launch_node_topk(goose_ctx* c, const __nv_bfloat16* logits, int rows, int V, int64_t ldl, int k,
-                             int32_t* argmax, int32_t* ids, float* vals, float* row_lse, cudaStream_t st);
+                             int32_t* argmax, int32_t* ids, float* vals, float* row_lse, cudaStream_t st,
+                             bool inputs_ready = false);
 cudaError_t launch_harvest_scatter(goose_ctx* c, const int32_t* row_tok, int rows, int table_rows, int k,
                                    const int32_t* ids, const float* vals, const float* row_lse,
                                    int32_t* adj_ids, float* adj_scores, cudaStream_t st);

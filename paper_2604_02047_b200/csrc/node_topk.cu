@@ -87,7 +87,8 @@ __global__ void __launch_bounds__(kTopkThreads, 1)
 node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items, int V, int64_t ldl, int k, int chunks,
                  u64* __restrict__ ws_cand, int32_t* __restrict__ row_counters,
                  int32_t* __restrict__ argmax, int32_t* __restrict__ ids, float* __restrict__ vals,
-                 float* __restrict__ row_lse, float2* __restrict__ ws_lse, int32_t* __restrict__ status) {
+                 float* __restrict__ row_lse, float2* __restrict__ ws_lse, int32_t* __restrict__ status,
+                 int inputs_ready) {
     extern __shared__ __align__(128) unsigned char s_stage[];   // kTopkStages x 64 KB
     __shared__ u64 s_full[kTopkStages];
     __shared__ float s_sum[32];
@@ -116,7 +117,12 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items, int 
     }
     if (tid < 32) s_list[tid] = 0;
     __syncthreads();
-    pdl_wait();
+    // inputs_ready: the caller guarantees that the logits were complete before the preceding kernel in the stream
+    // started (the whole-step call: that kernel is the attention merge, which neither reads nor writes them).  The
+    // CTA then streams and selects at once and only waits for the preceding kernel before its first write to global
+    // memory (outputs, cross-CTA scratch); otherwise it waits here, before its first read.
+    bool waited = inputs_ready == 0;
+    if (waited) pdl_wait();
     pdl_trigger();
 
     const unsigned short* lg = reinterpret_cast<const unsigned short*>(logits);
@@ -154,6 +160,7 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items, int 
 
     // warp 0: rank the pending item's candidates, merge them into the row's list, write what is complete
     auto finish_pending = [&]() {
+        if (!waited) { pdl_wait(); waited = true; }      // warp 0 does every global write of the CTA
         const int n_list = s_count;
         uint32_t mine = pend_mine;                       // lane r: the chunk's r-th winner
         if (!pend_has_mine) {
@@ -362,6 +369,7 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items, int 
         __syncthreads();
         if (s_abort) {
             // give up as one: report, wait (bounded) for this thread's copies still in flight, return
+            if (!waited) pdl_wait();                     // completion of this grid must imply that of the preceding one
             if (tid == 0) {
                 if (status) atomicOr(status, GOOSE_ST_TIMEOUT);
                 for (int jj = j; jj < issued; ++jj) topk_mbar_wait(&s_full[jj % kTopkStages], (uint32_t)(jj / kTopkStages) & 1u);
@@ -483,20 +491,21 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items, int 
         if (++chunk == chunks) { chunk = 0; ++row; }
     }
     if (warp == 0 && pend_chunk >= 0) finish_pending();  // the CTA's last item
+    if (!waited) pdl_wait();                             // (every CTA has at least one item, so warp 0 has waited)
 }
 
 namespace {
 template <int KCAP, bool LSE>
 cudaError_t launch_topk_inst(int grid, cudaStream_t st, const __nv_bfloat16* logits, long long items, int V, int64_t ldl,
                              int k, int chunks, u64* ws, int32_t* counters, int32_t* argmax, int32_t* ids, float* vals,
-                             float* row_lse, float2* ws_lse, int32_t* status) {
+                             float* row_lse, float2* ws_lse, int32_t* status, int inputs_ready) {
     return launch_pdl(node_topk_kernel<KCAP, LSE>, dim3(grid), dim3(kTopkThreads), kTopkSmem, st, logits, items, V, ldl, k,
-                      chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status);
+                      chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status, inputs_ready);
 }
 
 cudaError_t launch_topk_any(int num_sms, cudaStream_t st, const __nv_bfloat16* logits, int rows, int V, int64_t ldl, int k,
                             u64* ws, int32_t* counters, int32_t* argmax, int32_t* ids, float* vals, float* row_lse,
-                            float2* ws_lse, int32_t* status) {
+                            float2* ws_lse, int32_t* status, int inputs_ready) {
     const int chunks = (V + kTopkChunk - 1) / kTopkChunk;
     const long long items = (long long)rows * chunks;
     // every CTA gets q = ceil(items / SMs) items or one fewer; using the fewest CTAs that q allows loses no time and
@@ -504,10 +513,10 @@ cudaError_t launch_topk_any(int num_sms, cudaStream_t st, const __nv_bfloat16* l
     const long long q = (items + num_sms - 1) / num_sms;
     const int grid = (int)((items + q - 1) / q);
     if (row_lse)
-        return k <= 8 ? launch_topk_inst<8, true>(grid, st, logits, items, V, ldl, k, chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status)
-                      : launch_topk_inst<16, true>(grid, st, logits, items, V, ldl, k, chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status);
-    return k <= 8 ? launch_topk_inst<8, false>(grid, st, logits, items, V, ldl, k, chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status)
-                  : launch_topk_inst<16, false>(grid, st, logits, items, V, ldl, k, chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status);
+        return k <= 8 ? launch_topk_inst<8, true>(grid, st, logits, items, V, ldl, k, chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status, inputs_ready)
+                      : launch_topk_inst<16, true>(grid, st, logits, items, V, ldl, k, chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status, inputs_ready);
+    return k <= 8 ? launch_topk_inst<8, false>(grid, st, logits, items, V, ldl, k, chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status, inputs_ready)
+                  : launch_topk_inst<16, false>(grid, st, logits, items, V, ldl, k, chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status, inputs_ready);
 }
 }  // namespace
 
@@ -522,10 +531,11 @@ cudaError_t init_topk_kernel() {
 }
 
 cudaError_t launch_node_topk(goose_ctx* c, const __nv_bfloat16* logits, int rows, int V, int64_t ldl, int k,
-                             int32_t* argmax, int32_t* ids, float* vals, float* row_lse, cudaStream_t st) {
+                             int32_t* argmax, int32_t* ids, float* vals, float* row_lse, cudaStream_t st,
+                             bool inputs_ready) {
     if (rows == 0) return cudaSuccess;
     cudaError_t e = launch_topk_any(c->num_sms, st, logits, rows, V, ldl, k, c->topk_cand, c->row_counters, argmax, ids, vals,
-                                    row_lse, reinterpret_cast<float2*>(c->topk_lse_ws), c->status);
+                                    row_lse, reinterpret_cast<float2*>(c->topk_lse_ws), c->status, inputs_ready ? 1 : 0);
     c->launches++;
     return e;
 }
@@ -587,6 +597,6 @@ extern "C" int goose_node_topk_static(const void* logits, int rows, int V, int64
         return GOOSE_ECUDA;
     cudaError_t e = launch_topk_any(num_sms, st, static_cast<const __nv_bfloat16*>(logits), rows, V, ldl, k, scratch, counters,
                                     argmax, topk_ids, topk_vals, static_cast<float*>(nullptr), static_cast<float2*>(nullptr),
-                                    static_cast<int32_t*>(nullptr));
+                                    static_cast<int32_t*>(nullptr), 0);
     return e == cudaSuccess ? GOOSE_OK : GOOSE_ECUDA;
 }

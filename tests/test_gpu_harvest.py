@@ -62,6 +62,15 @@ def test_harvest_long_rows_and_row_stride(goose, oracle):
     _check(goose, oracle, const, 8, [1, 2], 40000)
 
 
+def test_harvest_more_items_than_sms(goose, oracle):
+    """Rows of three chunks, more items than SMs: the row log-sum-exp is merged over chunks inside a CTA and over CTAs."""
+    rng = np.random.default_rng(31)
+    rows, V, k = 200, 70000, 8
+    bits = synth.f32_to_bf16_bits((rng.standard_normal((rows, V)) * 3).astype(np.float32))
+    tok = rng.permutation(V)[:rows].astype(np.int32)
+    _check(goose, oracle, bits, k, tok, V, V=V)
+
+
 def test_harvest_argument_errors(goose):
     from paper_2604_02047_b200 import binding
     lg = torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda")

@@ -192,6 +192,23 @@ def test_topk_special_rows(goose, oracle):
     _check_topk(goose, oracle, rows, 8)
 
 
+@pytest.mark.parametrize("rows,V,k", [(100, 100000, 8), (333, 32000, 8), (150, 70000, 16), (1000, 40000, 5), (149, 32768, 8)])
+def test_topk_more_items_than_sms(goose, oracle, rows, V, k):
+    """More (row, 32768-element chunk) items than SMs: every CTA of the persistent kernel walks several items, rows longer
+    than a chunk fall across the CTAs' ranges (merged by the last CTA to arrive), and a few constant rows send single
+    items of a CTA down the exact slow path (more than 1024 elements tied at the threshold)."""
+    rng = np.random.default_rng([rows, V, k])
+    ldl = (V + 7) // 8 * 8
+    x = rng.standard_normal((rows, ldl), dtype=np.float32)
+    x[::3] = np.round(x[::3] * 4) / 4                          # every third row coarse: exact ties within and across chunks
+    bits = synth.f32_to_bf16_bits(x)
+    bits[:, V:] = 0x7F00                                       # huge values in the padding must be ignored
+    bits[rows // 2, :V] = 0x4000                               # constant rows
+    bits[rows - 1, :V] = 0xBF80
+    bits[rows // 3, : V // 2] = 0x4100                         # first half constant and above everything else
+    _check_topk(goose, oracle, bits, k, V=V)
+
+
 # ------------------------------------------------------------------ accept
 def test_accept_random_trees(goose, oracle):
     rng = np.random.default_rng(3)

@@ -83,6 +83,8 @@ cudaError_t launch_kv_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc
 // Fused form used by goose_verify_step: the acceptance walk (Algorithm 3) and the compaction in one launch.
 // Every CTA redoes the walk of its sequence with warp 0 (a handful of warp reductions) instead of waiting for
 // a separate kernel; CTA (0, 0, s) publishes path / accept_len / bonus / new_ctx.
+// parent[], draft_tok[], ctx_len[] and row_off[] are inputs of the step, complete before its first kernel started, so
+// they are read before the dependency wait; argmax[] (the top-k kernel's result) and the cache rows are read after it.
 __global__ void __launch_bounds__(kCompactThreads)
 accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __restrict__ row_off,
                       const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ draft_tok,
@@ -96,41 +98,47 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
     const int which = blockIdx.y;                        // 0 = K, 1 = V
     const int col = blockIdx.x * kCompactThreads + threadIdx.x;
     const bool publisher = blockIdx.x == 0 && which == 0;
-    pdl_wait();
-    pdl_trigger();
     // rows this sequence owns must lie inside the cache: never form an address from unchecked device data
     const int ctx0 = ctx_len[s];
     const int64_t r0 = row_off[s];
     const bool bad_rows = ctx0 < 0 || r0 < 0 || r0 + ctx0 + B > kv_rows;
+    constexpr int kPer = kMaxB / 32;
+    int my_par[kPer], my_tok[kPer];
+    bool bad = false;
     if (threadIdx.x < 32) {
         const int lane = threadIdx.x;
         const int32_t* par = parent + (size_t)s * B;
         const int32_t* tok = draft_tok + (size_t)s * B;
-        const int32_t* am = argmax + (size_t)s * B;
-        constexpr int kPer = kMaxB / 32;
-        int my_par[kPer];
-        bool my_match[kPer];
-        bool bad = false;
 #pragma unroll
         for (int t = 0; t < kPer; ++t) {
             const int c = lane + 32 * t;
             my_par[t] = -2;
-            my_match[t] = false;
+            my_tok[t] = -1;
             if (c < B) {
                 const int pp = par[c];
                 my_par[t] = pp;
+                my_tok[t] = tok[c];
                 bad |= (c == 0) ? (pp != -1) : (pp < 0 || pp >= c);
             }
         }
         bad = __any_sync(0xFFFFFFFFu, bad);
         for (int c = lane; c < B; c += 32) s_path[c] = (c == 0) ? 0 : -1;
+    }
+    pdl_wait();
+    pdl_trigger();
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x;
+        const int32_t* am = argmax + (size_t)s * B;
+        bool my_match[kPer];
+#pragma unroll
+        for (int t = 0; t < kPer; ++t) my_match[t] = false;
         __syncwarp();
         int v = 0, len = 0;
         if (!bad) {
 #pragma unroll
             for (int t = 0; t < kPer; ++t) {
                 const int c = lane + 32 * t;
-                if (c >= 1 && c < B) my_match[t] = (tok[c] == am[my_par[t]]);
+                if (c >= 1 && c < B) my_match[t] = (my_tok[t] == am[my_par[t]]);
             }
             for (int step = 0; step < B - 1; ++step) {
                 int cand = 0x7FFFFFFF;

@@ -136,14 +136,16 @@ int goose_harvest(goose_ctx* ctx, const void* logits, int rows, int V, int64_t l
  * of its device memory up front and treats a later cudaMalloc as an error, or a plug-in that is called
  * at a point where entering the allocator (and the implicit device synchronisation it can cause) is not
  * allowed.  goose_create allocates, so such callers cannot use goose_node_topk.  This variant computes
- * exactly the same result with the same kernel; its only scratch (the per-chunk winners and arrival
- * counters used when a row is longer than 32768 elements) is a fixed array of about 2 MiB that is part
- * of the library image, so every GPU that loads the library holds it until the process exits.
+ * exactly the same result with the same kernel; its only scratch (the partial winners and arrival
+ * counters used when the 32768-element chunks of a long row are handled by several thread blocks) is a
+ * fixed array of about 2 MiB that is part of the library image, so every GPU that loads the library holds
+ * it until the process exits.
  *   - Arguments, layouts and results as goose_node_topk, all data pointers on the CURRENT device;
  *     rows <= GOOSE_STATIC_TOPK_MAX_ROWS, otherwise GOOSE_EINVAL (nothing is enqueued).
  *   - It calls no cudaMalloc / cudaFree and no allocating library routine.  The first call on each
- *     device looks up the device address of the array (cudaGetSymbolAddress, with that device current);
- *     make that first call outside any stream capture.
+ *     device looks up the device address of the array (cudaGetSymbolAddress, with that device current),
+ *     reads the device's multiprocessor count and sets the kernel's shared-memory attribute; make that
+ *     first call outside any stream capture.
  *   - All calls share the one array, which keeps the contents of the previous call; the counters it
  *     needs at zero are cleared on `stream` before the kernel.  Two calls whose kernels may overlap on
  *     the GPU (different streams, no dependency between them) race on the array: serialise them.      */

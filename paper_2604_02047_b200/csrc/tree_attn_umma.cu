@@ -4,23 +4,25 @@
 // Work = all (sequence, head, 128-key tile) items in sequence-major order, dealt to the CTAs
 // (one per SM) in contiguous ranges, so every SM streams the same number of K/V bytes.  A run of
 // items of one head inside a CTA's range is a "segment"; a segment that covers its whole head
-// writes the bf16 output directly, any other segment writes an fp32 partial (unnormalised O, running
-// max m, running sum l) to the workspace, and a small second kernel (tree_attn_combine_kernel, spread
+// writes the bf16 output directly, any other segment writes a partial (O / l as fp16, running max m and
+// running sum l as fp32) to the workspace, and a small second kernel (tree_attn_combine_kernel, spread
 // over all SMs) merges the partials of every head that was split.
 //
 // Roles (192 threads):
 //   warp 0, lane 0   TMA producer: Q of the segment, then K and V tiles into a ring of 32 KB stages
-//   warp 1, lane 0   MMA issuer:   S = Q K^T into TMEM (double buffered), O += P V into TMEM
+//   warp 1, lane 0   MMA issuer:   S = Q K^T into TMEM (double buffered), O += P V into TMEM with P read
+//                                  from tensor memory
 //   warps 2..5       softmax:      one query row per thread (TMEM lane = row): S from TMEM, ancestor
-//                                  mask on the tiles that reach the tree rows, exp2, P (bf16) into
-//                                  shared memory in the canonical 128-byte-swizzled K-major layout,
-//                                  lazy rescaling of O in TMEM, epilogue (output or partial).
+//                                  mask on the tiles that reach the tree rows, exp2, P (bf16) written back
+//                                  over the first 64 columns of the S buffer it came from, lazy rescaling
+//                                  of O in TMEM, epilogue (output or partial).
 // All B <= 128 query rows ride in one M = 128 MMA; rows >= B compute on don't-care data and are
 // never written out.  Grouped-query attention (H query heads over Hkv key/value heads, g = H / Hkv) stacks the g
 // query heads of a group into the same M tile -- row r = (node r / g, group member r % g) -- so a K/V tile is
 // streamed once per group; when B * g > 128 the nodes are cut into M tiles of floor(128 / g) nodes and the K/V of a
-// head is streamed once per M tile.  A "head" of the work list below is one (M tile, key/value head) pair.  The tree part of the mask (Sec. 4 Stage 1: a node attends to the prefix and to
-// its root-to-node ancestors) is a per-row 128-bit ancestor set built from parent[].
+// head is streamed once per M tile.  A "head" of the work list below is one (M tile, key/value head) pair.
+// The tree part of the mask (Sec. 4 Stage 1: a node attends to the prefix and to its root-to-node ancestors) is a
+// per-row 128-bit ancestor set built from parent[].
 //
 // Every wait in this file is bounded: when a wait runs out of polls the CTA raises an abort flag,
 // sets GOOSE_ST_TIMEOUT, drains its own copies in flight (again bounded), frees its TMEM and returns.

@@ -20,7 +20,7 @@ def _tree(rng, B, kind):
 # (H, Hkv, B): group sizes 1..16, trees that fill the 128-row tile exactly, leave it ragged, or need several tiles
 # (B * g > 128), and a group size that does not divide 128
 GQA_SHAPES = [(8, 2, 32), (8, 2, 16), (8, 2, 33), (8, 2, 128), (6, 2, 50), (16, 1, 20), (4, 4, 20), (2, 1, 64),
-              (2, 1, 65), (32, 8, 32), (10, 2, 26), (12, 4, 1)]
+              (2, 1, 65), (32, 8, 32), (10, 2, 26), (12, 4, 1), (16, 1, 128), (64, 4, 128)]   # last two: the limits
 
 
 @pytest.mark.parametrize("impl", _impls(), ids=_impl_ids())

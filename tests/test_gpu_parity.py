@@ -172,7 +172,8 @@ def test_topk_generator_logits_and_ties(goose, oracle):
 
 
 @pytest.mark.parametrize("V,ldl,k", [(1, 8, 1), (5, 8, 5), (100, 104, 8), (8191, 8192, 8), (8192, 8192, 16),
-                                      (8193, 8200, 8), (32001, 32008, 10), (151936, 151936, 16)])
+                                      (8193, 8200, 8), (32001, 32008, 10), (151936, 151936, 16),
+                                      (262144, 262144, 16), (262143, 262144, 3)])   # the vocabulary limit
 def test_topk_sizes(goose, oracle, V, ldl, k):
     rng = np.random.default_rng(V)
     bits = synth.f32_to_bf16_bits(rng.standard_normal((7, ldl), dtype=np.float32))

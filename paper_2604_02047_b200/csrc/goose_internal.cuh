@@ -56,6 +56,26 @@ namespace goose {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Bounded mbarrier wait, shared by every kernel that waits on asynchronous copies or tensor-core commits.
+// Returns 0 when the barrier phase completed, 1 when `*abort_flag` was raised by another thread of the CTA meanwhile,
+// 2 when `limit_cycles` SM cycles passed (the caller raises the flag, records GOOSE_ST_TIMEOUT and unwinds).
+__device__ __forceinline__ bool mbar_try_wait_parity(unsigned long long* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"((uint32_t)__cvta_generic_to_shared(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ int mbar_wait_bounded(unsigned long long* bar, uint32_t parity, long long limit_cycles,
+                                                 volatile int* abort_flag) {
+    if (mbar_try_wait_parity(bar, parity)) return 0;
+    const long long t0 = clock64();
+    for (;;) {
+        if (*abort_flag) return 1;
+        if (mbar_try_wait_parity(bar, parity)) return 0;
+        if (clock64() - t0 > limit_cycles) return 2;
+    }
+}
+
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
                               Args&&... args) {

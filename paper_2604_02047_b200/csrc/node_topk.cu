@@ -64,20 +64,6 @@ __device__ __forceinline__ u64 warp_max_u64(u64 v) {
 
 namespace {
 __device__ __forceinline__ uint32_t topk_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ bool topk_mbar_try(u64* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(topk_smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-// bounded wait: false when the limit passes without the barrier completing
-__device__ __forceinline__ bool topk_mbar_wait(u64* bar, uint32_t parity) {
-    if (topk_mbar_try(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (clock64() - t0 < kTopkWaitCycles)
-        if (topk_mbar_try(bar, parity)) return true;
-    return false;
-}
 }  // namespace
 
 // LSE = true additionally returns the row's log-sum-exp (for the softmax scores of the harvest): the second
@@ -328,7 +314,7 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items, int 
         const int n_valid = min(kTopkChunk, V - base);
         const unsigned char* sp = s_stage + st * kTopkStageBytes;
         // a wait that runs out raises the CTA's abort flag; everybody learns of it behind the next barrier
-        const bool have = topk_mbar_wait(&s_full[st], (uint32_t)(j / kTopkStages) & 1u);
+        const bool have = mbar_wait_bounded(&s_full[st], (uint32_t)(j / kTopkStages) & 1u, kTopkWaitCycles, &s_abort) == 0;
         if (!have) s_abort = 1;
 
         // ---- phase 1: 32 values per thread into registers (element (it, e) of thread tid sits at chunk offset
@@ -372,7 +358,9 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items, int 
             if (!waited) pdl_wait();                     // completion of this grid must imply that of the preceding one
             if (tid == 0) {
                 if (status) atomicOr(status, GOOSE_ST_TIMEOUT);
-                for (int jj = j; jj < issued; ++jj) topk_mbar_wait(&s_full[jj % kTopkStages], (uint32_t)(jj / kTopkStages) & 1u);
+                volatile int no_abort = 0;               // draining ignores the abort flag
+                for (int jj = j; jj < issued; ++jj)
+                    mbar_wait_bounded(&s_full[jj % kTopkStages], (uint32_t)(jj / kTopkStages) & 1u, kTopkWaitCycles, &no_abort);
             }
             return;
         }

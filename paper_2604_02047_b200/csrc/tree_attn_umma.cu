@@ -869,7 +869,16 @@ bounded_wait_selftest_kernel(int32_t* __restrict__ status, long long limit_cycle
     __syncwarp();
     // the other lanes see the abort flag at once, as the other roles of the attention kernel would
     if (threadIdx.x != 0) ok = mbar_wait_limit(&hd, &hd.pv_done, 0, status, limit_cycles);
-    if (threadIdx.x == 1) result[0] = ok ? 1 : 0;         // 0 expected: the wait reported failure, the kernel returns
+    // the shared primitive the top-k kernel waits with: 1 (aborted) with the raised flag, 2 (timed out) with a clear one
+    __shared__ volatile int no_flag;
+    if (threadIdx.x == 1) no_flag = 0;
+    __syncwarp();
+    int bad = 0;
+    if (threadIdx.x == 1) {
+        bad |= mbar_wait_bounded(&hd.pv_done, 0, limit_cycles, &hd.abort_flag) != 1;
+        bad |= mbar_wait_bounded(&hd.pv_done, 0, limit_cycles, &no_flag) != 2;
+        result[0] = (ok ? 1 : 0) | (bad ? 2 : 0);          // 0 expected: every wait reported failure, the kernel returns
+    }
 }
 
 cudaError_t launch_bounded_wait_selftest(goose_ctx* c, long long limit_cycles, int32_t* result, cudaStream_t st) {

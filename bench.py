@@ -233,6 +233,11 @@ def run_ours(args, x, cfg, rank, world, local_rank):
         d = reps[i % R]
         g.harvest(d["logits"], x.k, d["draft_tok"].view(-1), adj_ids, adj_scores)
 
+    def step_harvest(i):     # the step and the harvest of its logits in one call (the logits are read once)
+        d, o = reps[i % R], outs[i % R]
+        g.verify_step_harvest(d["q"], d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], d["parent"], d["draft_tok"],
+                              d["logits"], x.k, x.scale, adj_ids, adj_scores, outs=o)
+
     with torch.cuda.stream(stream):
         for i in range(max(3, args.warmup)):
             step(i)
@@ -251,6 +256,7 @@ def run_ours(args, x, cfg, rank, world, local_rank):
         g_attn, _ = capture(attn)
         g_topk, _ = capture(topk)
         g_harv, _ = capture(harvest)
+        g_sh, _ = capture(step_harvest)
 
         def time_graph(gr, rounds):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -286,6 +292,8 @@ def run_ours(args, x, cfg, rank, world, local_rank):
             topk_ms = time_graph(g_topk, attn_rounds) / (attn_rounds * R)
             time_graph(g_harv, 1)
             harv_ms = time_graph(g_harv, attn_rounds) / (attn_rounds * R)
+            time_graph(g_sh, 1)
+            sh_ms = time_graph(g_sh, attn_rounds) / (attn_rounds * R)
         clocks = clk.summary()
     value, ms_per_step = aggregate_steps_per_s(args.steps, local_ms, world, dev)
 
@@ -345,6 +353,7 @@ def run_ours(args, x, cfg, rank, world, local_rank):
                      "traffic": NCU_TRAFFIC_BYTES.get(cfg.name), "algorithmic_bytes": ab["attn"],
                      "us_per_launch": attn_ms * 1e3},
         "kernels": {"tree_attn_us": attn_ms * 1e3, "node_topk_us": topk_ms * 1e3, "harvest_us": harv_ms * 1e3,
+                    "step_with_harvest_us": sh_ms * 1e3,
                     "node_topk_gbs": ab["topk"] / (topk_ms * 1e-3) / 1e9,
                     "step_gbs": ab["total"] / (ms_per_step * 1e-3) / 1e9,
                     "step_frac_of_peak": ab["total"] / (ms_per_step * 1e-3) / 1e9 / peak},

@@ -193,6 +193,20 @@ int goose_verify_step_gqa(goose_ctx* ctx, const void* q, void* k_cache, void* v_
                           int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
                           void* stream);
 
+/* The whole step plus the harvest of its logits (Algorithm 2: every cycle verifies a tree and harvests the forward's
+ * logits, rejected branches included): as goose_verify_step_gqa, and additionally row_lse fp32 [S*B] and the update
+ * of the adjacency table as in goose_harvest with row_tok = draft_tok (a node's logits row predicts the successor of
+ * that node's own draft token; rows with a negative token, e.g. padding nodes, are skipped).  The logits are read
+ * once: the top-k pass that feeds the acceptance walk also returns the log-sum-exp.  topk_vals is required.
+ * With row_lse, adj_ids and adj_scores all NULL (table_rows ignored) this is goose_verify_step_gqa.             */
+int goose_verify_step_harvest(goose_ctx* ctx, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
+                              const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
+                              const int32_t* draft_tok, const void* logits, int64_t ldl,
+                              int S, int B, int H, int Hkv, int D, int V, int k, float scale,
+                              void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
+                              int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
+                              float* row_lse, int table_rows, int32_t* adj_ids, float* adj_scores, void* stream);
+
 /* Host-buffer variant of the whole step (the end-to-end call).  The prefix KV cache stays on the
  * device (k_cache / v_cache are device pointers, state carried from step to step); everything a
  * step consumes or produces is in HOST memory (pinned memory makes the copies asynchronous):

@@ -22,6 +22,7 @@ EXPORTS = [
     "goose_verify_step_host", "goose_last_status", "goose_launch_count", "goose_node_topk_static", "goose_harvest",
     "goose_build_spine_tree", "goose_pad_tree", "goose_context_match", "goose_spine_ratio_tier", "goose_spine_ema",
     "goose_selftest_bounded_wait", "goose_tree_attn_gqa", "goose_verify_step_gqa", "goose_verify_step_host_gqa",
+    "goose_verify_step_harvest",
 ]
 
 ATTN_AUTO, ATTN_MMA, ATTN_UMMA = 0, 1, 2
@@ -268,6 +269,28 @@ class Goose:
             _p(outs["out"]), _p(outs.get("lse")), _p(outs["argmax"]), _p(outs["topk_ids"]), _p(outs["topk_vals"]),
             _p(outs["path"]), _p(outs["accept_len"]), _p(outs["bonus"]), _p(outs["new_ctx_len"]), _stream()),
             "goose_verify_step_gqa")
+        return outs
+
+    def verify_step_harvest(self, q, k_cache, v_cache, row_off, ctx_len, parent, draft_tok, logits, k: int, scale: float,
+                            adj_ids, adj_scores, outs: Optional[dict] = None, V: Optional[int] = None) -> dict:
+        """The whole step plus the harvest of its logits into the adjacency table (updated in place); multi-head or
+        grouped-query (Hkv is read from the caches' shape).  ``outs`` gains ``row_lse`` [S*B]."""
+        S, B, H, D = q.shape
+        Hkv = _kv_heads(k_cache, v_cache)
+        _dev(adj_ids, torch.int32, "adj_ids"); _dev(adj_scores, torch.float32, "adj_scores")
+        ldl = logits.shape[1]
+        V = ldl if V is None else V
+        if outs is None:
+            outs = self.alloc_step_outputs(S, B, H, D, k, q.device)
+        if "row_lse" not in outs:
+            outs["row_lse"] = torch.empty(S * B, dtype=torch.float32, device=q.device)
+        _check(self.lib.goose_verify_step_harvest(
+            self.h, _p(q), _p(k_cache), _p(v_cache), ctypes.c_int64(k_cache.shape[0]), _p(row_off), _p(ctx_len),
+            _p(parent), _p(draft_tok), _p(logits), ctypes.c_int64(ldl), ctypes.c_int(S), ctypes.c_int(B),
+            ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D), ctypes.c_int(V), ctypes.c_int(k), ctypes.c_float(scale),
+            _p(outs["out"]), _p(outs.get("lse")), _p(outs["argmax"]), _p(outs["topk_ids"]), _p(outs["topk_vals"]),
+            _p(outs["path"]), _p(outs["accept_len"]), _p(outs["bonus"]), _p(outs["new_ctx_len"]), _p(outs["row_lse"]),
+            ctypes.c_int(adj_ids.shape[0]), _p(adj_ids), _p(adj_scores), _stream()), "goose_verify_step_harvest")
         return outs
 
     def verify_step_host_gqa(self, k_cache, v_cache, h_q, h_k_new, h_v_new, h_row_off, h_ctx_len, h_parent,

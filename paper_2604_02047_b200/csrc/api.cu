@@ -235,7 +235,21 @@ int goose_verify_step_gqa(goose_ctx* c, const void* q, void* k_cache, void* v_ca
                           void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
                           int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
                           void* stream) {
+    return goose_verify_step_harvest(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, draft_tok, logits, ldl, S, B,
+                                     H, Hkv, D, V, k, scale, out, lse, argmax, topk_ids, topk_vals, path, accept_len, bonus,
+                                     new_ctx_len, nullptr, 0, nullptr, nullptr, stream);
+}
+
+int goose_verify_step_harvest(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
+                              const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
+                              const int32_t* draft_tok, const void* logits, int64_t ldl,
+                              int S, int B, int H, int Hkv, int D, int V, int k, float scale,
+                              void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
+                              int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
+                              float* row_lse, int table_rows, int32_t* adj_ids, float* adj_scores, void* stream) {
     // validate everything before enqueueing anything
+    const bool harvest = row_lse || adj_ids || adj_scores;
+    if (harvest && (!row_lse || !adj_ids || !adj_scores || !topk_vals || table_rows < 1)) return GOOSE_EINVAL;
     int rc = check_shape(c, S, B, H, D);
     if (rc) return rc;
     if (Hkv < 1 || H % Hkv != 0 || H / Hkv > GOOSE_MAX_GROUP) return GOOSE_EINVAL;
@@ -250,10 +264,12 @@ int goose_verify_step_gqa(goose_ctx* c, const void* q, void* k_cache, void* v_ca
                              stream);
     if (rc) return rc;
     // the logits are an input of the step: complete before the attention kernels above started, which do not touch
-    // them -- so the top-k kernel may read them while the attention merge is still running
+    // them -- so the top-k kernel may read them while the attention merge is still running.  With a harvest it also
+    // returns every row's log-sum-exp (one pass over the logits serves the walk and the table).
     if (S > 0) {
         cudaError_t et = goose::launch_node_topk(c, (const __nv_bfloat16*)logits, S * B, V, ldl, k, argmax, topk_ids, topk_vals,
-                                                 nullptr, static_cast<cudaStream_t>(stream), /*inputs_ready=*/true);
+                                                 harvest ? row_lse : nullptr, static_cast<cudaStream_t>(stream),
+                                                 /*inputs_ready=*/true);
         if (et != cudaSuccess) return cuda_fail(et);
     }
     // acceptance walk + compaction in one launch (same results as goose_accept followed by goose_kv_compact)
@@ -261,6 +277,13 @@ int goose_verify_step_gqa(goose_ctx* c, const void* q, void* k_cache, void* v_ca
                                                  draft_tok, parent, argmax, S, B, Hkv, kv_rows, path, accept_len, bonus,
                                                  new_ctx_len, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(e);
+    if (harvest && S > 0) {
+        // every logits row predicts the successor of its node's own draft token (padding nodes carry negative tokens
+        // and are skipped); the scatter comes last so that it does not delay the walk and the compaction
+        e = goose::launch_harvest_scatter(c, draft_tok, S * B, table_rows, k, topk_ids, topk_vals, row_lse, adj_ids, adj_scores,
+                                          static_cast<cudaStream_t>(stream));
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
     return GOOSE_OK;
 }
 

@@ -108,9 +108,9 @@ def test_goose_loop_is_lossless_and_keeps_the_cache_consistent():
         kn, vn = model.kv_rows(tok_t, torch.from_numpy(ctx + depth).cuda())
         k_cache[ctx:ctx + B] = kn; v_cache[ctx:ctx + B] = vn
         q = kn.unsqueeze(0).contiguous()                                   # any finite queries
-        o = g.verify_step(q, k_cache, v_cache, row_off, ctx_len, par_t.view(1, B).contiguous(),
-                          torch.from_numpy(tok).cuda().view(1, B), logits, K, scale)
-        g.harvest(logits, K, torch.from_numpy(tok).cuda(), adj_ids, adj_sc)
+        # one call per cycle: verify the tree and harvest the forward's logits (read once) into the table
+        o = g.verify_step_harvest(q, k_cache, v_cache, row_off, ctx_len, par_t.view(1, B).contiguous(),
+                                  torch.from_numpy(tok).cuda().view(1, B), logits, K, scale, adj_ids, adj_sc)
         torch.cuda.synchronize()
         assert torch.isfinite(o["out"].float()).all() and not g.last_status(1).any()
         L = int(o["accept_len"].item()); path = o["path"].cpu().numpy()[0]

@@ -71,6 +71,39 @@ def test_harvest_more_items_than_sms(goose, oracle):
     _check(goose, oracle, bits, k, tok, V, V=V)
 
 
+def test_step_with_harvest_equals_step_then_harvest(oracle):
+    """goose_verify_step_harvest reads the logits once; its step outputs equal goose_verify_step's and its table equals
+    goose_harvest's with row_tok = draft_tok, which in turn equals the oracle's."""
+    from paper_2604_02047_b200 import binding, build
+    build.build()
+    g = binding.Goose(max_S=4, max_B=128, max_H=64)
+    for x in (synth.make_config(0, seed=3),
+              synth.make_inputs(3, 8, 20, [100, 7, 260], [synth.kary_tree(20, 3), synth.chain_tree(20), synth.star_tree(20)],
+                                V=40000, seed=4, Hkv=2)):
+        x.draft_tok[0, 1] = -5                                         # a padding-style token: its row is skipped
+        d1, d2 = binding.to_device(x), binding.to_device(x)
+        step = g.verify_step if x.Hkv == x.H else g.verify_step_gqa
+        o1 = step(d1["q"], d1["k_cache"], d1["v_cache"], d1["row_off"], d1["ctx_len"], d1["parent"], d1["draft_tok"],
+                  d1["logits"], x.k, x.scale)
+        ids1 = torch.full((x.V, x.k), -7, dtype=torch.int32, device="cuda"); sc1 = torch.full((x.V, x.k), -1.0, device="cuda")
+        g.harvest(d1["logits"], x.k, d1["draft_tok"].view(-1), ids1, sc1)
+        ids2 = torch.full((x.V, x.k), -7, dtype=torch.int32, device="cuda"); sc2 = torch.full((x.V, x.k), -1.0, device="cuda")
+        o2 = g.verify_step_harvest(d2["q"], d2["k_cache"], d2["v_cache"], d2["row_off"], d2["ctx_len"], d2["parent"],
+                                   d2["draft_tok"], d2["logits"], x.k, x.scale, ids2, sc2)
+        torch.cuda.synchronize()
+        assert not g.last_status(x.S).any()
+        for key in ("out", "argmax", "topk_ids", "topk_vals", "path", "accept_len", "bonus", "new_ctx_len"):
+            assert torch.equal(o1[key], o2[key]), key
+        assert torch.equal(d1["k_cache"], d2["k_cache"]) and torch.equal(d1["v_cache"], d2["v_cache"])
+        assert torch.equal(ids1, ids2) and torch.equal(sc1, sc2)
+        rids, rsc, rlse = oracle.harvest(x.logits, x.k, x.draft_tok.reshape(-1), np.full((x.V, x.k), -7, np.int32),
+                                         np.full((x.V, x.k), -1.0, np.float64))
+        assert np.array_equal(ids2.cpu().numpy(), rids)
+        assert np.abs(sc2.cpu().numpy() - rsc).max() <= 1e-5 * max(1.0, np.abs(rsc).max())
+        assert np.abs(o2["row_lse"].cpu().numpy() - rlse).max() <= 2e-5 * max(1.0, np.abs(rlse).max())
+    g.close()
+
+
 def test_harvest_argument_errors(goose):
     from paper_2604_02047_b200 import binding
     lg = torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda")

@@ -272,18 +272,14 @@ int goose_verify_step_harvest(goose_ctx* c, const void* q, void* k_cache, void* 
                                                  /*inputs_ready=*/true);
         if (et != cudaSuccess) return cuda_fail(et);
     }
-    // acceptance walk + compaction in one launch (same results as goose_accept followed by goose_kv_compact)
+    // acceptance walk + compaction in one launch (same results as goose_accept followed by goose_kv_compact); with a
+    // harvest the launch also carries the table scatter: every logits row predicts the successor of its node's own draft
+    // token (padding nodes carry negative tokens and are skipped)
     cudaError_t e = goose::launch_accept_compact(c, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, row_off, ctx_len,
                                                  draft_tok, parent, argmax, S, B, Hkv, kv_rows, path, accept_len, bonus,
-                                                 new_ctx_len, static_cast<cudaStream_t>(stream));
+                                                 new_ctx_len, static_cast<cudaStream_t>(stream), table_rows, k, topk_ids,
+                                                 topk_vals, row_lse, harvest ? adj_ids : nullptr, adj_scores);
     if (e != cudaSuccess) return cuda_fail(e);
-    if (harvest && S > 0) {
-        // every logits row predicts the successor of its node's own draft token (padding nodes carry negative tokens
-        // and are skipped); the scatter comes last so that it does not delay the walk and the compaction
-        e = goose::launch_harvest_scatter(c, draft_tok, S * B, table_rows, k, topk_ids, topk_vals, row_lse, adj_ids, adj_scores,
-                                          static_cast<cudaStream_t>(stream));
-        if (e != cudaSuccess) return cuda_fail(e);
-    }
     return GOOSE_OK;
 }
 

@@ -105,7 +105,10 @@ cudaError_t launch_kv_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc
 cudaError_t launch_accept_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* row_off,
                                   const int32_t* ctx_len, const int32_t* draft_tok, const int32_t* parent,
                                   const int32_t* argmax, int S, int B, int H, int64_t kv_rows, int32_t* path,
-                                  int32_t* accept_len, int32_t* bonus, int32_t* new_ctx, cudaStream_t st);
+                                  int32_t* accept_len, int32_t* bonus, int32_t* new_ctx, cudaStream_t st,
+                                  int table_rows = 0, int k = 0, const int32_t* topk_ids = nullptr,
+                                  const float* topk_vals = nullptr, const float* row_lse = nullptr,
+                                  int32_t* adj_ids = nullptr, float* adj_scores = nullptr);
 cudaError_t launch_tree_attn_mma(goose_ctx* c, const __nv_bfloat16* q, const __nv_bfloat16* kc,
                                  const __nv_bfloat16* vc, int64_t kv_rows, const int64_t* row_off, const int32_t* ctx_len,
                                  const int32_t* parent, int S, int B, int H, int Hkv, float scale,

@@ -85,16 +85,50 @@ cudaError_t launch_kv_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc
 // a separate kernel; CTA (0, 0, s) publishes path / accept_len / bonus / new_ctx.
 // parent[], draft_tok[], ctx_len[] and row_off[] are inputs of the step, complete before its first kernel started, so
 // they are read before the dependency wait; argmax[] (the top-k kernel's result) and the cache rows are read after it.
+// With a harvest (adj_ids != NULL) the launch carries a third block role, blockIdx.y == 2: one warp per logits row of the
+// sequence writes that row's top-k ids and softmax scores to adjacency-table row draft_tok[row] unless a later row of the
+// call carries the same token -- the rule of harvest_scatter_kernel, decided here before the wait (tokens are inputs).
 __global__ void __launch_bounds__(kCompactThreads)
 accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __restrict__ row_off,
                       const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ draft_tok,
                       const int32_t* __restrict__ parent, const int32_t* __restrict__ argmax,
                       int B, int row_vec, int64_t kv_rows, int32_t* __restrict__ path,
                       int32_t* __restrict__ accept_len, int32_t* __restrict__ bonus, int32_t* __restrict__ new_ctx,
-                      int32_t* __restrict__ status) {
+                      int32_t* __restrict__ status,
+                      int rows_total, int table_rows, int k, const int32_t* __restrict__ topk_ids,
+                      const float* __restrict__ topk_vals, const float* __restrict__ row_lse,
+                      int32_t* __restrict__ adj_ids, float* __restrict__ adj_scores) {
     __shared__ int s_path[kMaxB];
     __shared__ int s_len;
     const int s = blockIdx.z;
+    if (blockIdx.y == 2) {
+        // ---- harvest scatter role
+        const int lane = threadIdx.x & 31;
+        const int i = blockIdx.x * (kCompactThreads / 32) + (threadIdx.x >> 5);   // node of sequence s
+        const size_t r = (size_t)s * B + i;
+        int tok = -1;
+        bool write = false;
+        if (i < B) {
+            tok = draft_tok[r];
+            if (tok >= 0 && tok < table_rows) {
+                bool later = false;                        // does a later row carry the same token?
+                for (int j = (int)r + 1 + lane; j < rows_total; j += 32) later |= (draft_tok[j] == tok);
+                write = !__any_sync(0xFFFFFFFFu, later);
+            }
+        }
+        pdl_wait();
+        pdl_trigger();
+        if (write && lane < k) {
+            adj_ids[(size_t)tok * k + lane] = topk_ids[r * k + lane];
+            adj_scores[(size_t)tok * k + lane] = expf(topk_vals[r * k + lane] - row_lse[r]);
+        }
+        return;
+    }
+    if ((int)blockIdx.x * kCompactThreads >= row_vec) {   // the grid is as wide as its widest role: nothing to copy here
+        pdl_wait();
+        pdl_trigger();
+        return;
+    }
     const int which = blockIdx.y;                        // 0 = K, 1 = V
     const int col = blockIdx.x * kCompactThreads + threadIdx.x;
     const bool publisher = blockIdx.x == 0 && which == 0;
@@ -187,12 +221,21 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
 cudaError_t launch_accept_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* row_off,
                                   const int32_t* ctx_len, const int32_t* draft_tok, const int32_t* parent,
                                   const int32_t* argmax, int S, int B, int H, int64_t kv_rows, int32_t* path,
-                                  int32_t* accept_len, int32_t* bonus, int32_t* new_ctx, cudaStream_t st) {
+                                  int32_t* accept_len, int32_t* bonus, int32_t* new_ctx, cudaStream_t st,
+                                  int table_rows, int k, const int32_t* topk_ids, const float* topk_vals,
+                                  const float* row_lse, int32_t* adj_ids, float* adj_scores) {
     if (S == 0) return cudaSuccess;
     int row_vec = H * kHeadDim * 2 / 16;
-    dim3 grid((row_vec + kCompactThreads - 1) / kCompactThreads, 2, S);
+    int gx = (row_vec + kCompactThreads - 1) / kCompactThreads;
+    const bool scatter = adj_ids != nullptr;
+    if (scatter) {
+        const int sx = (B + kCompactThreads / 32 - 1) / (kCompactThreads / 32);   // one warp per logits row
+        if (sx > gx) gx = sx;
+    }
+    dim3 grid(gx, scatter ? 3 : 2, S);
     cudaError_t e = launch_pdl(accept_compact_kernel, grid, dim3(kCompactThreads), 0, st, kc, vc, row_off, ctx_len,
-                               draft_tok, parent, argmax, B, row_vec, kv_rows, path, accept_len, bonus, new_ctx, c->status);
+                               draft_tok, parent, argmax, B, row_vec, kv_rows, path, accept_len, bonus, new_ctx, c->status,
+                               S * B, table_rows, k, topk_ids, topk_vals, row_lse, adj_ids, adj_scores);
     c->launches++;
     return e;
 }

@@ -111,3 +111,37 @@ def test_harvest_argument_errors(goose):
     with pytest.raises(binding.GooseError):
         goose.harvest(lg, 17, tok, torch.zeros((64, 17), dtype=torch.int32, device="cuda"),
                       torch.zeros((64, 17), dtype=torch.float32, device="cuda"))
+
+
+def test_step_with_harvest_argument_errors():
+    """A harvest needs all of row_lse, adj_ids, adj_scores and topk_vals; nothing is enqueued otherwise."""
+    import ctypes
+    from paper_2604_02047_b200 import binding, build
+    build.build()
+    g = binding.Goose(max_S=1, max_B=128, max_H=64)
+    x = synth.make_config(0, seed=5)
+    d = binding.to_device(x)
+    o = g.alloc_step_outputs(x.S, x.B, x.H, x.D, x.k, "cuda")
+    lse = torch.empty(x.S * x.B, dtype=torch.float32, device="cuda")
+    ids = torch.zeros((x.V, x.k), dtype=torch.int32, device="cuda"); sc = torch.zeros((x.V, x.k), device="cuda")
+    P = binding._p
+
+    def call(row_lse, adj_ids, adj_sc, vals, table_rows):
+        return g.lib.goose_verify_step_harvest(
+            g.h, P(d["q"]), P(d["k_cache"]), P(d["v_cache"]), ctypes.c_int64(d["k_cache"].shape[0]), P(d["row_off"]),
+            P(d["ctx_len"]), P(d["parent"]), P(d["draft_tok"]), P(d["logits"]), ctypes.c_int64(x.V), ctypes.c_int(x.S),
+            ctypes.c_int(x.B), ctypes.c_int(x.H), ctypes.c_int(x.H), ctypes.c_int(128), ctypes.c_int(x.V), ctypes.c_int(x.k),
+            ctypes.c_float(x.scale), P(o["out"]), None, P(o["argmax"]), P(o["topk_ids"]), P(vals), P(o["path"]),
+            P(o["accept_len"]), P(o["bonus"]), P(o["new_ctx_len"]), P(row_lse), ctypes.c_int(table_rows), P(adj_ids), P(adj_sc),
+            ctypes.c_void_p(torch.cuda.current_stream().cuda_stream))
+
+    n0 = g.launch_count()
+    assert call(lse, ids, None, o["topk_vals"], x.V) == -1          # scores missing
+    assert call(None, ids, sc, o["topk_vals"], x.V) == -1           # row_lse missing
+    assert call(lse, ids, sc, None, x.V) == -1                      # topk_vals missing
+    assert call(lse, ids, sc, o["topk_vals"], 0) == -1              # empty table
+    assert g.launch_count() == n0                                   # nothing was enqueued
+    assert call(lse, ids, sc, o["topk_vals"], x.V) == 0
+    assert call(None, None, None, None, 0) == 0                     # no harvest: the plain step, topk_vals optional
+    torch.cuda.synchronize()
+    g.close()

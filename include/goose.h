@@ -216,7 +216,10 @@ int goose_verify_step_harvest(goose_ctx* ctx, const void* q, void* k_cache, void
  *   out: h_out bf16 [S][B][H][D]; h_argmax [S*B]; h_topk_ids [S*B][k]; h_topk_vals [S*B][k] or NULL;
  *        h_path [S][B]; h_accept_len, h_bonus, h_new_ctx_len [S]
  * Copies in, runs goose_verify_step, copies out, and synchronises `stream` before returning.
- * Device staging buffers are allocated inside the context on first use and grow on demand.      */
+ * The logits (most of the bytes, needed by the top-k only) are uploaded on a stream of the context's own while the
+ * attention kernels run; the small arrays travel through one pinned block of the context, one copy each way.
+ * Device and pinned staging buffers, that stream and its events are created inside the context on first use and
+ * grow on demand; calls on one context must not overlap.                                                     */
 int goose_verify_step_host(goose_ctx* ctx, void* k_cache, void* v_cache, int64_t kv_rows,
                            const void* h_q, const void* h_k_new, const void* h_v_new,
                            const int64_t* h_row_off, const int32_t* h_ctx_len,

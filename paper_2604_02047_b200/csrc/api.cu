@@ -115,6 +115,10 @@ int goose_destroy(goose_ctx* c) {
     cudaSetDevice(c->device);
     cudaFree(c->partials); cudaFree(c->head_counters); cudaFree(c->topk_cand);
     cudaFree(c->row_counters); cudaFree(c->topk_lse_ws); cudaFree(c->status); cudaFree(c->selftest_word); cudaFree(c->stage);
+    if (c->pin) cudaFreeHost(c->pin);
+    if (c->side) cudaStreamDestroy(c->side);
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+    if (c->ev_logits) cudaEventDestroy(c->ev_logits);
     delete c;
     return GOOSE_OK;
 }
@@ -240,6 +244,23 @@ int goose_verify_step_gqa(goose_ctx* c, const void* q, void* k_cache, void* v_ca
                                      new_ctx_len, nullptr, 0, nullptr, nullptr, stream);
 }
 
+}  // extern "C"
+
+namespace {
+// The step's launches.  logits_ready (may be NULL): an event the stream has to wait for before the top-k, for callers
+// that produce the logits next to the attention kernels (the host-buffer call uploads them on a side stream).
+int enqueue_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
+                 const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
+                 const int32_t* draft_tok, const void* logits, int64_t ldl,
+                 int S, int B, int H, int Hkv, int D, int V, int k, float scale,
+                 void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
+                 int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
+                 float* row_lse, int table_rows, int32_t* adj_ids, float* adj_scores, void* stream,
+                 cudaEvent_t logits_ready);
+}  // namespace
+
+extern "C" {
+
 int goose_verify_step_harvest(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
                               const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
                               const int32_t* draft_tok, const void* logits, int64_t ldl,
@@ -247,6 +268,22 @@ int goose_verify_step_harvest(goose_ctx* c, const void* q, void* k_cache, void* 
                               void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
                               int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
                               float* row_lse, int table_rows, int32_t* adj_ids, float* adj_scores, void* stream) {
+    return enqueue_step(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, draft_tok, logits, ldl, S, B, H, Hkv, D, V, k,
+                        scale, out, lse, argmax, topk_ids, topk_vals, path, accept_len, bonus, new_ctx_len, row_lse, table_rows,
+                        adj_ids, adj_scores, stream, nullptr);
+}
+
+}  // extern "C"
+
+namespace {
+int enqueue_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
+                 const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
+                 const int32_t* draft_tok, const void* logits, int64_t ldl,
+                 int S, int B, int H, int Hkv, int D, int V, int k, float scale,
+                 void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
+                 int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
+                 float* row_lse, int table_rows, int32_t* adj_ids, float* adj_scores, void* stream,
+                 cudaEvent_t logits_ready) {
     // validate everything before enqueueing anything
     const bool harvest = row_lse || adj_ids || adj_scores;
     if (harvest && (!row_lse || !adj_ids || !adj_scores || !topk_vals || table_rows < 1)) return GOOSE_EINVAL;
@@ -267,6 +304,8 @@ int goose_verify_step_harvest(goose_ctx* c, const void* q, void* k_cache, void* 
     // them -- so the top-k kernel may read them while the attention merge is still running.  With a harvest it also
     // returns every row's log-sum-exp (one pass over the logits serves the walk and the table).
     if (S > 0) {
+        // (with logits_ready the kernel cannot start before the event, so reading ahead of its own wait stays safe)
+        if (logits_ready) GOOSE_CUDA(cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), logits_ready, 0));
         cudaError_t et = goose::launch_node_topk(c, (const __nv_bfloat16*)logits, S * B, V, ldl, k, argmax, topk_ids, topk_vals,
                                                  harvest ? row_lse : nullptr, static_cast<cudaStream_t>(stream),
                                                  /*inputs_ready=*/true);
@@ -282,6 +321,9 @@ int goose_verify_step_harvest(goose_ctx* c, const void* q, void* k_cache, void* 
     if (e != cudaSuccess) return cuda_fail(e);
     return GOOSE_OK;
 }
+}  // namespace
+
+extern "C" {
 
 int goose_verify_step_host(goose_ctx* c, void* k_cache, void* v_cache, int64_t kv_rows,
                            const void* h_q, const void* h_k_new, const void* h_v_new,
@@ -344,7 +386,32 @@ int goose_verify_step_host_gqa(goose_ctx* c, void* k_cache, void* v_cache, int64
         c->stage_bytes = off;
     }
     char* d = static_cast<char*>(c->stage);
+    // one-off per context: the side stream and its events, and the pinned block for the small arrays
+    if (!c->side) {
+        GOOSE_CUDA(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking));
+        GOOSE_CUDA(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
+        GOOSE_CUDA(cudaEventCreateWithFlags(&c->ev_logits, cudaEventDisableTiming));
+    }
+    const size_t in_bytes = o_tok + rows * 4 - o_rowoff;           // row_off | ctx_len | parent | draft_tok (padded as above)
+    const size_t out_bytes = o_newctx + (size_t)S * 4 - o_argmax;  // argmax | ids | vals | path | accept_len | bonus | new_ctx
+    const size_t pin_need = up(in_bytes) + out_bytes;
+    if (pin_need > c->pin_bytes) {
+        GOOSE_CUDA(cudaStreamSynchronize(st));
+        if (c->pin) cudaFreeHost(c->pin);
+        c->pin = nullptr; c->pin_bytes = 0;
+        if (cudaHostAlloc(&c->pin, pin_need, cudaHostAllocDefault) != cudaSuccess) { cudaGetLastError(); return GOOSE_ENOMEM; }
+        c->pin_bytes = pin_need;
+    }
+    char* pin_in = static_cast<char*>(c->pin);
+    char* pin_out = pin_in + up(in_bytes);
     const size_t row_bytes = (size_t)Hkv * D * 2;       // one cache row
+
+    // what the attention needs first: the small arrays (one copy through the pinned block), Q and the tree rows of K/V
+    memcpy(pin_in + (o_rowoff - o_rowoff), h_row_off, (size_t)S * 8);
+    memcpy(pin_in + (o_ctx - o_rowoff), h_ctx_len, (size_t)S * 4);
+    memcpy(pin_in + (o_parent - o_rowoff), h_parent, rows * 4);
+    memcpy(pin_in + (o_tok - o_rowoff), h_draft_tok, rows * 4);
+    GOOSE_CUDA(cudaMemcpyAsync(d + o_rowoff, pin_in, in_bytes, cudaMemcpyHostToDevice, st));
     GOOSE_CUDA(cudaMemcpyAsync(d + o_q, h_q, n_q, cudaMemcpyHostToDevice, st));
     for (int s = 0; s < S; ++s) {
         size_t dst = (size_t)(h_row_off[s] + h_ctx_len[s]) * row_bytes;
@@ -353,26 +420,32 @@ int goose_verify_step_host_gqa(goose_ctx* c, void* k_cache, void* v_cache, int64
         GOOSE_CUDA(cudaMemcpyAsync((char*)v_cache + dst, (const char*)h_v_new + (size_t)s * B * row_bytes,
                                    (size_t)B * row_bytes, cudaMemcpyHostToDevice, st));
     }
-    GOOSE_CUDA(cudaMemcpyAsync(d + o_logits, h_logits, rows * V * 2, cudaMemcpyHostToDevice, st));
-    GOOSE_CUDA(cudaMemcpyAsync(d + o_rowoff, h_row_off, S * 8, cudaMemcpyHostToDevice, st));
-    GOOSE_CUDA(cudaMemcpyAsync(d + o_ctx, h_ctx_len, S * 4, cudaMemcpyHostToDevice, st));
-    GOOSE_CUDA(cudaMemcpyAsync(d + o_parent, h_parent, rows * 4, cudaMemcpyHostToDevice, st));
-    GOOSE_CUDA(cudaMemcpyAsync(d + o_tok, h_draft_tok, rows * 4, cudaMemcpyHostToDevice, st));
-    rc = goose_verify_step_gqa(c, d + o_q, k_cache, v_cache, kv_rows, (const int64_t*)(d + o_rowoff),
-                               (const int32_t*)(d + o_ctx), (const int32_t*)(d + o_parent), (const int32_t*)(d + o_tok),
-                               d + o_logits, V, S, B, H, Hkv, D, V, k, scale, d + o_out, nullptr, (int32_t*)(d + o_argmax),
-                               (int32_t*)(d + o_ids), (float*)(d + o_vals), (int32_t*)(d + o_path),
-                               (int32_t*)(d + o_alen), (int32_t*)(d + o_bonus), (int32_t*)(d + o_newctx), stream);
-    if (rc) return rc;
+    // the logits (most of the bytes, needed by the top-k only) go up on the side stream while the attention kernels run;
+    // the fork sits behind the copies above, so they have the host link to themselves and the attention starts first
+    GOOSE_CUDA(cudaEventRecord(c->ev_fork, st));
+    GOOSE_CUDA(cudaStreamWaitEvent(c->side, c->ev_fork, 0));
+    GOOSE_CUDA(cudaMemcpyAsync(d + o_logits, h_logits, rows * V * 2, cudaMemcpyHostToDevice, c->side));
+    GOOSE_CUDA(cudaEventRecord(c->ev_logits, c->side));
+    rc = enqueue_step(c, d + o_q, k_cache, v_cache, kv_rows, (const int64_t*)(d + o_rowoff),
+                      (const int32_t*)(d + o_ctx), (const int32_t*)(d + o_parent), (const int32_t*)(d + o_tok),
+                      d + o_logits, V, S, B, H, Hkv, D, V, k, scale, d + o_out, nullptr, (int32_t*)(d + o_argmax),
+                      (int32_t*)(d + o_ids), (float*)(d + o_vals), (int32_t*)(d + o_path),
+                      (int32_t*)(d + o_alen), (int32_t*)(d + o_bonus), (int32_t*)(d + o_newctx), nullptr, 0, nullptr, nullptr,
+                      stream, c->ev_logits);
+    if (rc) {
+        cudaStreamSynchronize(c->side);                  // nothing of this call may stay in flight behind an error
+        return rc;
+    }
     GOOSE_CUDA(cudaMemcpyAsync(h_out, d + o_out, n_q, cudaMemcpyDeviceToHost, st));
-    GOOSE_CUDA(cudaMemcpyAsync(h_argmax, d + o_argmax, rows * 4, cudaMemcpyDeviceToHost, st));
-    GOOSE_CUDA(cudaMemcpyAsync(h_topk_ids, d + o_ids, rows * k * 4, cudaMemcpyDeviceToHost, st));
-    if (h_topk_vals) GOOSE_CUDA(cudaMemcpyAsync(h_topk_vals, d + o_vals, rows * k * 4, cudaMemcpyDeviceToHost, st));
-    GOOSE_CUDA(cudaMemcpyAsync(h_path, d + o_path, rows * 4, cudaMemcpyDeviceToHost, st));
-    GOOSE_CUDA(cudaMemcpyAsync(h_accept_len, d + o_alen, S * 4, cudaMemcpyDeviceToHost, st));
-    GOOSE_CUDA(cudaMemcpyAsync(h_bonus, d + o_bonus, S * 4, cudaMemcpyDeviceToHost, st));
-    GOOSE_CUDA(cudaMemcpyAsync(h_new_ctx_len, d + o_newctx, S * 4, cudaMemcpyDeviceToHost, st));
+    GOOSE_CUDA(cudaMemcpyAsync(pin_out, d + o_argmax, out_bytes, cudaMemcpyDeviceToHost, st));   // the small results: one copy
     GOOSE_CUDA(cudaStreamSynchronize(st));
+    memcpy(h_argmax, pin_out + (o_argmax - o_argmax), rows * 4);
+    memcpy(h_topk_ids, pin_out + (o_ids - o_argmax), rows * k * 4);
+    if (h_topk_vals) memcpy(h_topk_vals, pin_out + (o_vals - o_argmax), rows * k * 4);
+    memcpy(h_path, pin_out + (o_path - o_argmax), rows * 4);
+    memcpy(h_accept_len, pin_out + (o_alen - o_argmax), (size_t)S * 4);
+    memcpy(h_bonus, pin_out + (o_bonus - o_argmax), (size_t)S * 4);
+    memcpy(h_new_ctx_len, pin_out + (o_newctx - o_argmax), (size_t)S * 4);
     return GOOSE_OK;
 }
 

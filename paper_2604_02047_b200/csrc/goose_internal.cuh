@@ -40,6 +40,10 @@ struct goose_ctx {
     // host staging for goose_verify_step_host
     void* stage;              // device buffer
     size_t stage_bytes;
+    void* pin;                // pinned host block: the small input arrays go up, the small results come down, in one copy each
+    size_t pin_bytes;
+    cudaStream_t side;        // the logits are uploaded here, next to the attention kernels
+    cudaEvent_t ev_fork, ev_logits;
     long long launches;
     void* encode_tiled;       // cuTensorMapEncodeTiled entry point (driver), resolved at create
 };

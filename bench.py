@@ -188,6 +188,55 @@ def run_reference(args, x, cfg_name):
 
 
 # ----------------------------------------------------------------------------- GPU legs
+def quick_step_timing(config_id, dev, steps, peak):
+    """Whole-step and attention timing of another workload of the table, same method as the main line (CUDA-graph replay
+    over rotating replicas, CUDA events), without the CPU and end-to-end legs: context for the main line, not a bench line."""
+    import torch
+    from paper_2604_02047_b200 import binding, synth
+    x = synth.make_config(config_id)
+    g = binding.Goose(max_S=x.S, max_B=128, max_H=max(64, x.H), device=dev.index)
+    base = binding.to_device(x, dev)
+    footprint = sum(t.numel() * t.element_size() for t in base.values())
+    R = int(max(2, min(64, -(-max(2 * L2_BYTES, 1 << 30) // footprint))))
+    reps = [base] + [{k: v.clone() for k, v in base.items()} for _ in range(R - 1)]
+    outs = [g.alloc_step_outputs(x.S, x.B, x.H, x.D, x.k, dev) for _ in range(R)]
+    stream = torch.cuda.Stream(device=dev)
+
+    def step(i):
+        d = reps[i % R]
+        g.verify_step(d["q"], d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], d["parent"], d["draft_tok"],
+                      d["logits"], x.k, x.scale, outs=outs[i % R])
+
+    def attn(i):
+        d = reps[i % R]
+        g.tree_attn(d["q"], d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], d["parent"], x.scale, out=outs[i % R]["out"])
+
+    res = {}
+    with torch.cuda.stream(stream):
+        for i in range(3):
+            step(i)
+        stream.synchronize()
+        for name, fn in (("step", step), ("attn", attn)):
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr, stream=stream, capture_error_mode="thread_local"):
+                for i in range(R):
+                    fn(i)
+            rounds = max(3, -(-steps // R))
+            for _ in range(2):
+                gr.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(rounds):
+                gr.replay()
+            e1.record(stream)
+            e1.synchronize()
+            res[name] = e0.elapsed_time(e1) / (rounds * R)       # ms per call
+    ab = synth.algorithmic_bytes(x.S, x.H, x.B, x.D, x.V, x.ctx_len, Hkv=x.Hkv)
+    g.close()
+    return {"steps_per_s": 1e3 / res["step"], "us_per_step": res["step"] * 1e3, "tree_attn_us": res["attn"] * 1e3,
+            "tree_attn_frac_of_peak": ab["attn"] / (res["attn"] * 1e-3) / 1e9 / peak}
+
+
 def run_ours(args, x, cfg, rank, world, local_rank):
     import torch
     from paper_2604_02047_b200 import binding, build, synth
@@ -362,6 +411,11 @@ def run_ours(args, x, cfg, rank, world, local_rank):
         cb = oracle_sample(x)
         line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
     g.close()
+    # context for the single-GPU default line: the other batch-1 workloads of the table, timed the same way
+    if rank == 0 and world == 1 and args.config == 3 and not args.no_others and not args.attn_impl:
+        del reps, outs, base
+        torch.cuda.empty_cache()
+        line["other_workloads"] = {synth.CONFIGS[cid].name: quick_step_timing(cid, dev, args.steps, peak) for cid in (1, 2)}
     if rank == 0:
         print(json.dumps(line))
 
@@ -377,6 +431,8 @@ def main():
     ap.add_argument("--attn-impl", choices=["mma", "umma"], default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-others", action="store_true",
+                    help="skip the short timings of the 7b and 13b workloads that the default line carries as context")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 

@@ -81,3 +81,50 @@ def test_attention_random_shapes(goose, oracle, seed):
                 assert np.abs(lse.cpu().numpy() - ref_lse).max() <= 3e-3, where
         finally:
             goose.set_attn_impl(binding.ATTN_AUTO)
+
+
+@pytest.mark.parametrize("seed", [31, 32])
+def test_step_with_harvest_random_shapes(oracle, seed):
+    """The whole step plus harvest on random batches (multi-head and grouped, 1-5 sequences, tree sizes 2-128, vocabularies
+    64-70000, k 1-16, a few padding-style negative tokens): every integer result and the compacted cache rows bit-exact,
+    table scores within 1e-5, attention within the usual bar."""
+    from paper_2604_02047_b200 import binding, build
+    build.build()
+    g = binding.Goose(max_S=8, max_B=128, max_H=64)
+    rng = np.random.default_rng(seed)
+    for _ in range(6):
+        Hkv = int(rng.choice([1, 2, 4, 8])); H = Hkv * int(rng.choice([1, 1, 2, 4]))
+        B = int(rng.integers(2, 129)); S = int(rng.integers(1, 6))
+        V = (int(rng.choice([64, 1000, 4096, 32000, 50000, 70000])) + 7) // 8 * 8
+        k = min(int(rng.integers(1, 17)), V)
+        ctxs = [int(rng.choice([0, rng.integers(1, 200), rng.integers(100, 1500)])) for _ in range(S)]
+        trees = [synth.spine_tree(rng, B, max(1, B // int(rng.integers(2, 6))), 3) for _ in range(S)]
+        x = synth.make_inputs(S, H, B, ctxs, [t[0] for t in trees], V=V, k=k, seed=int(rng.integers(1 << 30)), Hkv=Hkv,
+                              is_spine=[t[1] for t in trees], p_spine=0.8, p_branch=0.3)
+        for s in range(S):
+            for i in rng.integers(1, B, 2):
+                x.draft_tok[s, i] = -1 - int(i)                 # never matched, never harvested
+        where = "S=%d B=%d H=%d Hkv=%d V=%d k=%d ctx=%s" % (S, B, H, Hkv, V, k, ctxs)
+        d = binding.to_device(x)
+        ids = torch.full((V, k), -7, dtype=torch.int32, device="cuda"); sc = torch.full((V, k), -1.0, device="cuda")
+        o = g.verify_step_harvest(d["q"], d["k_cache"], d["v_cache"], d["row_off"], d["ctx_len"], d["parent"], d["draft_tok"],
+                                  d["logits"], k, x.scale, ids, sc)
+        torch.cuda.synchronize()
+        assert not g.last_status(S).any(), where
+        ram, rids, _ = oracle.node_topk(x.logits, k)
+        rp, rl, rb = oracle.accept(x.draft_tok, x.parent, ram.reshape(S, B))
+        rk, rv, rn = oracle.kv_compact(x.k_cache, x.v_cache, x.row_off, x.ctx_len, rp, rl)
+        hids, hsc, _ = oracle.harvest(x.logits, k, x.draft_tok.reshape(-1), np.full((V, k), -7, np.int32), np.full((V, k), -1.0))
+        ref, _ = oracle.tree_attn(x.q, x.k_cache, x.v_cache, x.row_off, x.ctx_len, x.parent, x.scale)
+        assert np.array_equal(o["argmax"].cpu().numpy(), ram) and np.array_equal(o["topk_ids"].cpu().numpy(), rids), where
+        assert np.array_equal(o["path"].cpu().numpy(), rp) and np.array_equal(o["accept_len"].cpu().numpy(), rl), where
+        assert np.array_equal(o["bonus"].cpu().numpy(), rb) and np.array_equal(o["new_ctx_len"].cpu().numpy(), rn), where
+        gk, gv = binding.bf16_to_bits(d["k_cache"]), binding.bf16_to_bits(d["v_cache"])
+        for s in range(S):
+            r0, n = int(x.row_off[s]), int(rn[s])
+            assert np.array_equal(gk[r0:r0 + n], rk[r0:r0 + n]) and np.array_equal(gv[r0:r0 + n], rv[r0:r0 + n]), where
+        assert np.array_equal(ids.cpu().numpy(), hids), where
+        assert np.all(np.abs(sc.cpu().numpy() - hsc) <= 1e-5 * np.abs(hsc) + 1e-9), where
+        got = o["out"].float().cpu().numpy().astype(np.float64)
+        assert attn_row_err(got, ref).max() <= ATTN_TOL, where
+    g.close()

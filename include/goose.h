@@ -21,7 +21,9 @@
  *     detected on the device: the affected sequence gets zero-filled / neutral outputs and a
  *     non-zero status word (goose_last_status); a kernel never traps and never spins without
  *     a bound.
- *   - A goose_ctx must not be used from two streams at once (its workspace is shared).
+ *   - A goose_ctx must not be used from two streams at once (its workspace is shared), and every call that takes
+ *     a context must be made with the context's device current (cudaSetDevice), otherwise GOOSE_EINVAL;
+ *     goose_verify_step_host, goose_last_status and goose_selftest_bounded_wait select the device themselves.
  *
  * Tree layout (Algorithm 1): node 0 is the anchor/root and counts towards B;
  * parent[0] = -1 and 0 <= parent[i] < i (topological order).  B <= GOOSE_MAX_B.
@@ -148,7 +150,11 @@ int goose_harvest(goose_ctx* ctx, const void* logits, int rows, int V, int64_t l
  *     first call outside any stream capture.
  *   - All calls share the one array, which keeps the contents of the previous call; the counters it
  *     needs at zero are cleared on `stream` before the kernel.  Two calls whose kernels may overlap on
- *     the GPU (different streams, no dependency between them) race on the array: serialise them.      */
+ *     the GPU (different streams, no dependency between them) race on the array: serialise them.
+ *   - There is no status word behind this entry point: should one of the kernel's bounded waits run out (a
+ *     copy that never completes), the call has already returned GOOSE_OK, the time-out is not reported, and
+ *     the rows concerned keep whatever argmax / topk_ids / topk_vals held before.  Callers that need the
+ *     report use goose_node_topk.                                                                        */
 int goose_node_topk_static(const void* logits, int rows, int V, int64_t ldl, int k,
                            int32_t* argmax, int32_t* topk_ids, float* topk_vals, void* stream);
 
@@ -166,7 +172,10 @@ int goose_accept(goose_ctx* ctx, const int32_t* draft_tok, const int32_t* parent
  * the accepted nodes' rows in path order directly after the prefix, in place:
  * row ctx_len[s]+j <- row ctx_len[s]+path[s][j] for j = 0..accept_len[s], for K and V;
  * new_ctx_len[s] = ctx_len[s] + 1 + accept_len[s].  Rows >= new_ctx_len[s] are unspecified after
- * the call.  path must be increasing (as goose_accept produces it).                              */
+ * the call.  path must be increasing (as goose_accept produces it).
+ * new_ctx_len must not overlap ctx_len (GOOSE_EINVAL): every thread block of the launch reads ctx_len[s]
+ * while one of them writes new_ctx_len[s].  To chain steps without a host round trip, alternate two
+ * arrays: step t+1 takes step t's new_ctx_len as its ctx_len and writes the other array.             */
 int goose_kv_compact(goose_ctx* ctx, void* k_cache, void* v_cache, int64_t kv_rows,
                      const int64_t* row_off, const int32_t* ctx_len, const int32_t* path,
                      const int32_t* accept_len, int S, int B, int H, int D,
@@ -174,7 +183,10 @@ int goose_kv_compact(goose_ctx* ctx, void* k_cache, void* v_cache, int64_t kv_ro
 
 /* The whole step on one stream, in data-flow order: tree attention, node top-k (rows = S*B),
  * acceptance walk, KV compaction (the last two share one launch).  Arguments and results as in the
- * four calls above.                                                                             */
+ * four calls above (new_ctx_len must not overlap ctx_len).  q, the caches' tree rows, parent, draft_tok,
+ * logits, ctx_len and row_off are INPUTS of the step: they must be complete in stream order before the
+ * call and nothing else may write them until the step is done; some kernels of the step read them
+ * ahead of their stream-order dependency on the step's earlier kernels.                              */
 int goose_verify_step(goose_ctx* ctx, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
                       const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
                       const int32_t* draft_tok, const void* logits, int64_t ldl,
@@ -273,7 +285,10 @@ float goose_spine_ema(float p_hat, int accepted_spine, int drafted_spine);
 
 /* Synchronise the device, copy the per-sequence status words (GOOSE_ST_* bits, OR-ed over all
  * calls since the last query) into host_status[0..S) (a HOST array) and clear them.
- * Returns GOOSE_ETIMEOUT if any word has GOOSE_ST_TIMEOUT set.  For tests and debugging.         */
+ * Returns GOOSE_ETIMEOUT if any word has GOOSE_ST_TIMEOUT set.  For tests and debugging.
+ * Recovery rule: a call whose kernel timed out leaves its outputs incomplete and the context's cross-block
+ * arrival counters half counted; this query is what resets them, so after a GOOSE_ST_TIMEOUT call it once
+ * before the context is used again.                                                               */
 int goose_last_status(goose_ctx* ctx, int32_t* host_status, int S);
 
 /* Self-test of the device-side time-out path.  Runs a one-warp kernel whose wait (the same bounded mbarrier wait

@@ -49,7 +49,7 @@ def lib() -> ctypes.CDLL:
         _lib.oracle_num_threads.restype = ctypes.c_int
         for name in ("oracle_tree_attn", "oracle_tree_attn_rows", "oracle_tree_attn_gqa", "oracle_tree_attn_rows_gqa",
                      "oracle_node_topk", "oracle_accept",
-                     "oracle_kv_compact", "oracle_check_parent", "oracle_harvest"):
+                     "oracle_kv_compact", "oracle_check_parent", "oracle_harvest", "oracle_ancestors"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
 
@@ -168,6 +168,20 @@ def kv_compact(k_cache, v_cache, row_off, ctx_len, path, accept_len
     if rc != 0:
         raise ValueError("oracle_kv_compact failed: rc=%d" % rc)
     return k_out, v_out, new_ctx
+
+
+def ancestors(parent) -> list:
+    """Ancestor sets A(i) (Sec. 4 Stage 1: root-to-node path, node included) of every node as bitmasks, bit j = node j."""
+    parent = _c(parent, np.int32).reshape(-1)
+    B = len(parent)
+    masks = []
+    for i in range(B):
+        vis = np.zeros(B, dtype=np.uint8)
+        rc = lib().oracle_ancestors(_ptr(parent, ctypes.c_int32), ctypes.c_int(B), ctypes.c_int(i), _ptr(vis, ctypes.c_uint8))
+        if rc != 0:
+            raise ValueError("oracle_ancestors failed: rc=%d (invalid parent[]?)" % rc)
+        masks.append(sum(1 << j for j in range(B) if vis[j]))
+    return masks
 
 
 def check_parent(parent) -> bool:

@@ -66,6 +66,12 @@ static int ancestors_of(const int32_t* parent, int B, int i, unsigned char* vis)
     return vis[0] ? 0 : -1;
 }
 
+/* The ancestor set of node i as the tests see it: vis[j] = 1 iff j in A(i), j = 0..B-1.  Same return codes. */
+int oracle_ancestors(const int32_t* parent, int B, int i, unsigned char* vis) {
+    if (B < 1 || i < 0 || i >= B) return -1;
+    return ancestors_of(parent, B, i, vis);
+}
+
 int oracle_check_parent(const int32_t* parent, int B) {
     if (B < 1 || parent[0] != -1) return -1;
     for (int i = 1; i < B; ++i)

@@ -22,8 +22,23 @@ int cuda_fail(cudaError_t e) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// new_ctx_len[] may not overlap ctx_len[]: every block of the compaction launch reads ctx_len[s] while one of them
+// writes new_ctx_len[s], so an in-place update would let late blocks move rows relative to the new length
+bool ctx_arrays_overlap(const int32_t* ctx_len, const int32_t* new_ctx_len, int S) {
+    const uintptr_t a = reinterpret_cast<uintptr_t>(ctx_len), b = reinterpret_cast<uintptr_t>(new_ctx_len);
+    const uintptr_t n = sizeof(int32_t) * (uintptr_t)(S > 0 ? S : 1);
+    return a < b + n && b < a + n;
+}
+
+// the context's workspace, kernel attributes and tensor maps belong to c->device: a stream-ordered call made with
+// another device current would fail at launch with an opaque CUDA error
+bool on_ctx_device(const goose_ctx* c) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == c->device;
+}
+
 int check_shape(const goose_ctx* c, int S, int B, int H, int D) {
-    if (!c) return GOOSE_EINVAL;
+    if (!c || !on_ctx_device(c)) return GOOSE_EINVAL;
     if (S < 0 || S > c->max_S) return GOOSE_EINVAL;
     if (B < 1 || B > c->max_B || B > GOOSE_MAX_B) return GOOSE_EINVAL;
     if (H < 1 || H > c->max_H) return GOOSE_EINVAL;
@@ -81,6 +96,7 @@ int goose_create(goose_ctx** out, int device, int max_S, int max_B, int max_H, i
     c->topk_cand_cap = (int64_t)c->topk_rows_cap * kTopkMaxChunks * GOOSE_MAX_K;
 
     bool ok = true;
+    cudaError_t setup_err = cudaSuccess;               // a failure that is not an allocation keeps its own code
     ok = ok && cudaMalloc(&c->partials, sizeof(float) * (size_t)c->n_slots * goose::kPartialFloats) == cudaSuccess;
     ok = ok && cudaMalloc(&c->head_counters, sizeof(int32_t) * (size_t)heads) == cudaSuccess;
     ok = ok && cudaMalloc(&c->topk_cand, sizeof(unsigned long long) * (size_t)c->topk_cand_cap) == cudaSuccess;
@@ -99,12 +115,13 @@ int goose_create(goose_ctx** out, int device, int max_S, int max_B, int max_H, i
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
             qres == cudaDriverEntryPointSuccess)
             c->encode_tiled = fn;
-        ok = goose::init_kernels(c) == cudaSuccess;
+        setup_err = goose::init_kernels(c);            // e.g. a device that is not sm_100: no kernel image
+        ok = setup_err == cudaSuccess;
     }
     if (!ok) {
         cudaGetLastError();
         goose_destroy(c);
-        return GOOSE_ENOMEM;
+        return setup_err != cudaSuccess ? cuda_fail(setup_err) : GOOSE_ENOMEM;
     }
     *out = c;
     return GOOSE_OK;
@@ -167,7 +184,7 @@ int goose_tree_attn_gqa(goose_ctx* c, const void* q, const void* k_cache, const 
 
 int goose_node_topk(goose_ctx* c, const void* logits, int rows, int V, int64_t ldl, int k,
                     int32_t* argmax, int32_t* topk_ids, float* topk_vals, void* stream) {
-    if (!c || !logits || !argmax || !topk_ids) return GOOSE_EINVAL;
+    if (!c || !on_ctx_device(c) || !logits || !argmax || !topk_ids) return GOOSE_EINVAL;
     if (rows < 0 || rows > c->topk_rows_cap) return GOOSE_EINVAL;
     if (V < 1 || V > GOOSE_MAX_V || ldl < V || (ldl & 7) != 0 || !aligned16(logits)) return GOOSE_EINVAL;
     if (k < 1 || k > GOOSE_MAX_K || k > V) return GOOSE_EINVAL;
@@ -180,7 +197,8 @@ int goose_node_topk(goose_ctx* c, const void* logits, int rows, int V, int64_t l
 int goose_harvest(goose_ctx* c, const void* logits, int rows, int V, int64_t ldl, int k, const int32_t* row_tok,
                   int table_rows, int32_t* adj_ids, float* adj_scores, int32_t* argmax, int32_t* topk_ids,
                   float* topk_vals, float* row_lse, void* stream) {
-    if (!c || !logits || !row_tok || !adj_ids || !adj_scores || !argmax || !topk_ids || !topk_vals || !row_lse)
+    if (!c || !on_ctx_device(c) || !logits || !row_tok || !adj_ids || !adj_scores || !argmax || !topk_ids || !topk_vals ||
+        !row_lse)
         return GOOSE_EINVAL;
     if (rows < 0 || rows > c->topk_rows_cap || table_rows < 1) return GOOSE_EINVAL;
     if (V < 1 || V > GOOSE_MAX_V || ldl < V || (ldl & 7) != 0 || !aligned16(logits)) return GOOSE_EINVAL;
@@ -197,7 +215,7 @@ int goose_harvest(goose_ctx* c, const void* logits, int rows, int V, int64_t ldl
 
 int goose_accept(goose_ctx* c, const int32_t* draft_tok, const int32_t* parent, const int32_t* argmax,
                  int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus, void* stream) {
-    if (!c || !draft_tok || !parent || !argmax || !path || !accept_len || !bonus) return GOOSE_EINVAL;
+    if (!c || !on_ctx_device(c) || !draft_tok || !parent || !argmax || !path || !accept_len || !bonus) return GOOSE_EINVAL;
     if (S < 0 || S > c->max_S || B < 1 || B > c->max_B) return GOOSE_EINVAL;
     cudaError_t e = goose::launch_accept(c, draft_tok, parent, argmax, S, B, path, accept_len, bonus,
                                          static_cast<cudaStream_t>(stream));
@@ -213,6 +231,7 @@ int goose_kv_compact(goose_ctx* c, void* k_cache, void* v_cache, int64_t kv_rows
     if (rc) return rc;
     if (!k_cache || !v_cache || !row_off || !ctx_len || !path || !accept_len || !new_ctx_len) return GOOSE_EINVAL;
     if (!aligned16(k_cache) || !aligned16(v_cache) || kv_rows < 1) return GOOSE_EINVAL;
+    if (ctx_arrays_overlap(ctx_len, new_ctx_len, S)) return GOOSE_EINVAL;
     cudaError_t e = goose::launch_kv_compact(c, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, row_off, ctx_len,
                                              path, accept_len, S, B, H, kv_rows, new_ctx_len,
                                              static_cast<cudaStream_t>(stream));
@@ -297,6 +316,7 @@ int enqueue_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int6
         return GOOSE_EINVAL;
     if (V < 1 || V > GOOSE_MAX_V || ldl < V || (ldl & 7) != 0 || k < 1 || k > GOOSE_MAX_K || k > V) return GOOSE_EINVAL;
     if ((long long)S * B > c->topk_rows_cap || kv_rows < 1 || kv_rows > 0x7FFFFFFFLL) return GOOSE_EINVAL;
+    if (ctx_arrays_overlap(ctx_len, new_ctx_len, S)) return GOOSE_EINVAL;
     rc = goose_tree_attn_gqa(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, S, B, H, Hkv, D, scale, out, lse,
                              stream);
     if (rc) return rc;
@@ -346,6 +366,8 @@ int goose_verify_step_host_gqa(goose_ctx* c, void* k_cache, void* v_cache, int64
                                void* h_out, int32_t* h_argmax, int32_t* h_topk_ids, float* h_topk_vals,
                                int32_t* h_path, int32_t* h_accept_len, int32_t* h_bonus,
                                int32_t* h_new_ctx_len, void* stream) {
+    if (!c) return GOOSE_EINVAL;
+    GOOSE_CUDA(cudaSetDevice(c->device));               // this call selects the context's device itself
     int rc = check_shape(c, S, B, H, D);
     if (rc) return rc;
     if (Hkv < 1 || H % Hkv != 0 || H / Hkv > GOOSE_MAX_GROUP) return GOOSE_EINVAL;
@@ -357,7 +379,6 @@ int goose_verify_step_host_gqa(goose_ctx* c, void* k_cache, void* v_cache, int64
     if (S == 0) return GOOSE_OK;
     for (int s = 0; s < S; ++s)
         if (h_row_off[s] < 0 || h_ctx_len[s] < 0 || h_row_off[s] + h_ctx_len[s] + B > kv_rows) return GOOSE_EINVAL;
-    GOOSE_CUDA(cudaSetDevice(c->device));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
     // staging layout (256-byte aligned pieces)
@@ -470,6 +491,12 @@ int goose_last_status(goose_ctx* c, int32_t* host_status, int S) {
     int rc = GOOSE_OK;
     for (int s = 0; s < S; ++s)
         if (host_status[s] & GOOSE_ST_TIMEOUT) rc = GOOSE_ETIMEOUT;
+    if (rc == GOOSE_ETIMEOUT) {
+        // a CTA that gave up never arrived at its row's / head's counter, and the CTAs that had arrived left it non-zero
+        // (only the last arriver resets it): clear them all, the device is idle here
+        GOOSE_CUDA(cudaMemset(c->head_counters, 0, sizeof(int32_t) * (size_t)c->max_S * (size_t)c->max_H));
+        GOOSE_CUDA(cudaMemset(c->row_counters, 0, sizeof(int32_t) * (size_t)c->topk_rows_cap));
+    }
     return rc;
 }
 

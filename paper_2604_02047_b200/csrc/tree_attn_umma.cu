@@ -28,7 +28,6 @@
 // sets GOOSE_ST_TIMEOUT, drains its own copies in flight (again bounded), frees its TMEM and returns.
 #include <cuda.h>
 #include <cuda_fp16.h>
-#include <cstdlib>
 
 #include "goose_internal.cuh"
 
@@ -56,24 +55,6 @@ constexpr int kCombineRound = 4;                 // partials merged per load rou
 constexpr int kPartHalfWords = 16 * 128 * 4;     // 32-bit words of the fp16 block
 constexpr int kUmmaPartFloats = kPartHalfWords + 2 * kMaxB;
 constexpr long long kWaitCycles = 2000000000ll;  // bound of every wait: about one second of SM clock
-
-#ifdef GOOSE_TRACE
-// Debug build only: per-CTA, per-role timestamp log (64 entries of tag<<56 | globaltimer ns per role).
-__device__ unsigned long long* g_trace = nullptr;
-__device__ __forceinline__ void trace_ev(int role, int& n, unsigned tag) {
-    if (g_trace && n < 64) {
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-        g_trace[((size_t)blockIdx.x * 3 + role) * 64 + n] = ((unsigned long long)tag << 56) | (t & 0x00FFFFFFFFFFFFFFull);
-        ++n;
-    }
-}
-#define TRACE(role, n, tag) trace_ev(role, n, tag)
-#define TRACE_DECL int tn = 0
-#else
-#define TRACE(role, n, tag) do { } while (0)
-#define TRACE_DECL do { } while (0)
-#endif
 
 struct Header {                                  // lives at the start of dynamic shared memory
     unsigned long long kv_full[kStages];
@@ -348,8 +329,6 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 Cursor cu; cu.seek(wk, w_begin);
                 uint32_t ring = 0, seg = 0;
                 bool ok = true;
-                TRACE_DECL;
-                TRACE(0, tn, 1);
                 while (ok && cu.w < w_end) {
                     const int64_t row0 = row_off[cu.s];
                     // Q of this segment
@@ -376,7 +355,6 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                             tma_load_3d_hint(dst, mp, &hd->kv_full[st], 0, hk, krow, pol_stream);
                             tma_load_3d_hint(dst + kHalfBytes, mp, &hd->kv_full[st], 64, hk, krow, pol_stream);
                             ++ring;
-                            TRACE(0, tn, 2);
                         }
                         cu.next(wk);
                     }
@@ -395,8 +373,6 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 Cursor cu; cu.seek(wk, w_begin);
                 uint32_t jg = 0, seg = 0;                  // CTA-global tile and segment counters
                 bool ok = true;
-                TRACE_DECL;
-                TRACE(1, tn, 1);
                 const uint32_t q_base = smem_u32(q_smem), kv_addr = smem_u32(kv_smem);
                 constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
 
@@ -417,7 +393,6 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                     }
                     umma_commit(&hd->kv_empty[st]);
                     umma_commit(&hd->pv_done);
-                    TRACE(1, tn, 3);
                     return true;
                 };
 
@@ -441,7 +416,6 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                                      idesc_qk, kk > 0 ? 1u : 0u);
                         }
                         umma_commit(&hd->s_full[jg & 1]);
-                        TRACE(1, tn, 2);
                         umma_commit(&hd->kv_empty[st]);
                         if (jg > j_first) ok = issue_pv(jg - 1, jg - 1 == j_first);
                         ++jg;
@@ -467,8 +441,6 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
             int cur_s = -1, cur_mt = -1;
             bool bad = false;
             uint32_t anc[4] = {0, 0, 0, 0};
-            TRACE_DECL;
-            if (sm_tid == 0) TRACE(2, tn, 1);
 
             while (ok && cu.w < w_end) {
                 const int s0 = cu.s, h0 = cu.h, T = cu.T;
@@ -531,7 +503,6 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                     ok = mbar_wait(hd, &hd->s_full[jg & 1], (jg >> 1) & 1, status);
                     if (!ok) break;
                     tc_fence_after();
-                    if (sm_tid == 0 && seg_tiles < 2) TRACE(2, tn, 2);
                     float m_use = 0.f;
                     if (warp_has_rows) {
                         const uint32_t s_addr = tmem + kColS + (jg & 1) * 128 + lane_sel;
@@ -634,7 +605,6 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                     }
                     tc_fence_before();
                     mbar_arrive(&hd->p_ready);
-                    if (sm_tid == 0 && seg_tiles < 2) TRACE(2, tn, 3);
                     ++jg;
                     ++seg_tiles;
                     cu.next(wk);
@@ -645,7 +615,6 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 ok = mbar_wait(hd, &hd->pv_done, (jg - 1) & 1, status);
                 if (!ok) break;
                 tc_fence_after();
-                if (sm_tid == 0) TRACE(2, tn, 4);
                 const int n_tiles_seg = seg_tiles;
                 const bool whole_head = (t_first == 0) && (n_tiles_seg == T);
                 if (warp_has_rows) {
@@ -697,9 +666,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                         part[kPartHalfWords + row] = bad ? (t_first == 0 ? 0.f : -INFINITY) : m_run;
                         part[kPartHalfWords + kMaxB + row] = bad ? (t_first == 0 ? 1.f : 0.f) : l_run;
                     }
-                    if (sm_tid == 0) TRACE(2, tn, 5);
                 }
-                if (sm_tid == 0) TRACE(2, tn, 8);
                 ++seg;
             }
         }
@@ -845,13 +812,6 @@ bool make_map(void* fn, CUtensorMap* map, const void* base, int64_t rows, int H,
 
 }  // namespace
 
-#ifdef GOOSE_TRACE
-extern "C" int goose_debug_set_trace(void* dev_ptr) {
-    unsigned long long* p = static_cast<unsigned long long*>(dev_ptr);
-    return (int)cudaMemcpyToSymbol(g_trace, &p, sizeof p);
-}
-#endif
-
 // Self-test of the bounded-wait path: one warp waits on a barrier that nothing ever completes, with a short
 // limit.  The wait must give up, set GOOSE_ST_TIMEOUT in status[0] and let the kernel return normally, the same way
 // a stalled pipeline of the attention kernel would.  Nothing here can hang: the only loop is the bounded wait.
@@ -923,9 +883,6 @@ cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __
                                kv_rows, scale * kLog2e, c->partials, c->status, out, lse);
     c->launches++;
     if (e != cudaSuccess) return e;
-#ifdef GOOSE_TRACE
-    if (getenv("GOOSE_SKIP_COMBINE")) return e;       // debug build only: time the main kernel alone
-#endif
     dim3 cgrid((nb * g + 31) / 32, n_mt * Hkv, S);
     const float* parts = c->partials;
     e = launch_pdl(grouped ? tree_attn_combine_kernel<true> : tree_attn_combine_kernel<false>, cgrid,

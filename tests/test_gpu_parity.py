@@ -11,6 +11,11 @@ from paper_2604_02047_b200 import synth
 pytestmark = pytest.mark.gpu
 
 ATTN_TOL = 1e-2
+# Optional log-sum-exp output: the benchmark spec states no tolerance for it, this one is derived.  lse = m + ln(l), with the
+# scores accumulated in fp32 by the tensor core and l = the fp32 sum of up to n = 40 960 terms exp2(s - m) per row (the
+# longest fixture): the worst case of that sum is a relative error of n * 2^-24 = 2.4e-3 in l, i.e. the same absolute
+# error in ln(l); ex2.approx / log2f add about 1e-6.  The bound is absolute because lse may be near zero.
+LSE_TOL = 3e-3
 
 
 @pytest.fixture(scope="module")
@@ -59,7 +64,7 @@ def _check_attn_full(goose, oracle, x, impl):
     ref, ref_lse = oracle.tree_attn(x.q, x.k_cache, x.v_cache, x.row_off, x.ctx_len, x.parent, x.scale)
     err = attn_row_err(out, ref)
     assert err.max() <= ATTN_TOL, (err.max(), np.unravel_index(err.argmax(), err.shape))
-    assert np.abs(lse - ref_lse).max() <= 2e-3
+    assert np.abs(lse - ref_lse).max() <= LSE_TOL
 
 
 # ------------------------------------------------------------------ attention
@@ -100,7 +105,7 @@ def test_attention_extreme_partitions(goose, oracle, impl):
     ss, si, sh = np.zeros(8, np.int32), np.arange(8, dtype=np.int32), np.zeros(8, np.int32)
     ref, ref_lse = oracle.tree_attn_rows(x.q, x.k_cache, x.v_cache, x.row_off, x.ctx_len, x.parent, x.scale, ss, si, sh)
     assert not st.any() and attn_row_err(out[0, :, 0], ref).max() <= ATTN_TOL
-    assert np.abs(lse[0, :, 0] - ref_lse).max() <= 2e-3
+    assert np.abs(lse[0, :, 0] - ref_lse).max() <= LSE_TOL
     rng = np.random.default_rng(43)
     S = 16
     y = synth.make_inputs(S, 12, 5, rng.integers(0, 300, S), [synth.random_tree(rng, 5) for _ in range(S)], V=8,
@@ -325,7 +330,7 @@ def test_rows_outside_the_cache_are_flagged_and_nothing_is_moved(goose):
 
 
 # ------------------------------------------------------------------ whole step on the benchmark configs
-def _check_step(goose, oracle, x, n_rows=192, host=False):
+def _check_step(goose, oracle, x, n_rows=0, host=False):
     from paper_2604_02047_b200 import binding
     d = binding.to_device(x)
     if host:
@@ -357,14 +362,19 @@ def _check_step(goose, oracle, x, n_rows=192, host=False):
     for s in range(x.S):
         r0, n = int(x.row_off[s]), int(rn[s])
         assert np.array_equal(gk[r0:r0 + n], rk[r0:r0 + n]) and np.array_equal(gv[r0:r0 + n], rv[r0:r0 + n])
-    # attention: sampled (sequence, node, head) rows, always including node 0, the deepest node and the last node
-    rng = np.random.default_rng(1)
-    ss = rng.integers(0, x.S, n_rows); si = rng.integers(0, x.B, n_rows); sh = rng.integers(0, x.H, n_rows)
-    si[:3] = [0, x.B - 1, int(np.argmax(x.is_spine[ss[2]].cumsum() * x.is_spine[ss[2]]))]
-    ref, _ = oracle.tree_attn_rows(x.q, x.k_cache, x.v_cache, x.row_off, x.ctx_len, x.parent, x.scale, ss, si, sh)
-    got = o["out"].float().cpu().numpy().astype(np.float64)[ss, si, sh]
+    # attention: EVERY (sequence, node, head) row against the oracle (1.6 s of oracle time at 33b, about 11 s at batch16);
+    # n_rows > 0 asks for a sample instead (rows drawn uniformly, plus node 0, the last node and the deepest spine node)
+    got = o["out"].float().cpu().numpy().astype(np.float64)
+    if n_rows:
+        rng = np.random.default_rng(1)
+        ss = rng.integers(0, x.S, n_rows); si = rng.integers(0, x.B, n_rows); sh = rng.integers(0, x.H, n_rows)
+        si[:3] = [0, x.B - 1, int(np.argmax(x.is_spine[ss[2]].cumsum() * x.is_spine[ss[2]]))]
+        ref, _ = oracle.tree_attn_rows(x.q, x.k_cache, x.v_cache, x.row_off, x.ctx_len, x.parent, x.scale, ss, si, sh)
+        got = got[ss, si, sh]
+    else:
+        ref, _ = oracle.tree_attn(x.q, x.k_cache, x.v_cache, x.row_off, x.ctx_len, x.parent, x.scale, want_lse=False)
     err = attn_row_err(got, ref)
-    assert err.max() <= ATTN_TOL, err.max()
+    assert err.max() <= ATTN_TOL, (err.max(), np.unravel_index(err.argmax(), err.shape))
     return float(err.max())
 
 

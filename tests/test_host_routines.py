@@ -2,6 +2,7 @@
 import numpy as np
 import pytest
 
+from _golden import load_spine_tree_example
 from oracle import spine_tree as st
 
 
@@ -27,6 +28,16 @@ def test_build_spine_tree_matches_the_oracle(binding):
         otok, opar, osp, info = st.build_spine_tree(anchor, d.tolist(), adj, B, D, r, rho)
         assert n == len(otok) and ns == info["b_s"] + 1
         assert tok.tolist() == otok and par.tolist() == opar and sp.tolist() == osp
+
+
+def test_build_spine_tree_matches_the_hand_worked_example(binding):
+    """goose_build_spine_tree against the tree worked out by hand from Algorithm 1 (not against the oracle)."""
+    ex = load_spine_tree_example()
+    for D, tok, parent, n_spine in ex["cases"]:
+        gtok, gpar, gsp, n, ns = binding.build_spine_tree(ex["anchor"], ex["chain"], ex["adj"], ex["B"], D, ex["r"], ex["rho"])
+        assert n == len(tok) and ns == n_spine, D
+        assert gtok.tolist() == tok and gpar.tolist() == parent
+        assert gsp.tolist() == [True] * n_spine + [False] * (n - n_spine)
 
 
 def test_padding_nodes_can_never_be_accepted(binding, oracle):

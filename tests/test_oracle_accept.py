@@ -31,6 +31,7 @@ def _load_hand_example():
 def test_hand_example(oracle):
     ex = _load_hand_example()
     B = ex["B"]
+    assert oracle.ancestors(ex["parent"]) == ex["anc"]          # the ancestor sets behind the tree attention mask
     for name, am, path, alen, bonus in ex["cases"]:
         p, l, b = oracle.accept(ex["draft_tok"], ex["parent"], am)
         assert l[0] == alen and b[0] == bonus, name

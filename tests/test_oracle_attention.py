@@ -149,6 +149,14 @@ def test_invalid_parent_is_rejected(oracle):
     with pytest.raises(ValueError):
         oracle.tree_attn(x.q, x.k_cache, x.v_cache, x.row_off, x.ctx_len, bad, x.scale)
     assert not oracle.check_parent(bad) and oracle.check_parent(x.parent)
+    # every way parent[] can fail to be a rooted tree in topological order (parent[0] = -1, 0 <= parent[i] < i)
+    for bad in ([0, 0, 1], [-1, 1, 0], [-1, -1, 0], [-1, 0, 2], [-1, 0, 3], [1, 0, 0], [-2, 0, 1]):
+        assert not oracle.check_parent(np.array(bad, np.int32)), bad
+        with pytest.raises(ValueError):
+            oracle.ancestors(np.array(bad, np.int32))
+    for good in ([-1], [-1, 0], [-1, 0, 0, 2, 1, 4]):
+        assert oracle.check_parent(np.array(good, np.int32))
+    assert oracle.ancestors([-1, 0, 0, 2, 1, 4]) == [0b1, 0b11, 0b101, 0b1101, 0b10011, 0b110011]
 
 
 # ------------------------------------------------------------------ grouped-query attention

@@ -1,6 +1,7 @@
 """Pins for the host-side oracle: Algorithm 1 (BuildSpineTree), ContextMatch, spine-ratio tiers."""
 import numpy as np
 
+from _golden import load_spine_tree_example
 from oracle import spine_tree as st
 
 
@@ -57,6 +58,20 @@ def test_tree_invariants_on_random_tables():
         assert len(root_kids) <= info["b_r"]
         for i in range(1, b_s + 1):
             assert len([c for c in range(b_s + 1, n) if parent[c] == i]) <= info["a"][i - 1]
+
+
+def test_hand_worked_tree():
+    """The hand-worked example fixes what the invariants above leave open: the chain is cut to floor(B r) nodes, the
+    rank order of the attached successors, the duplicate skip taking the next-ranked entry without using up the
+    allocation, a_i = 0, and step 4 extending the leaves breadth first, in creation order, by their TOP-ranked successor
+    up to D nodes per branch."""
+    ex = load_spine_tree_example()
+    assert st.budget_split(len(ex["chain"]), ex["B"], ex["r"], ex["rho"]) == tuple(ex["budget"])
+    assert st.harmonic_allocation(ex["budget"][0], ex["budget"][2]) == ex["alloc"]
+    for D, tok, parent, n_spine in ex["cases"]:
+        otok, opar, ospine, info = st.build_spine_tree(ex["anchor"], ex["chain"], ex["adj"], ex["B"], D, ex["r"], ex["rho"])
+        assert otok == tok and opar == parent, D
+        assert ospine == [True] * n_spine + [False] * (len(tok) - n_spine) and info["a"] == ex["alloc"]
 
 
 def test_special_trees():

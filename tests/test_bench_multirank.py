@@ -61,3 +61,28 @@ def test_reference_arm_prints_one_contract_line():
     assert d["impl"] == "reference" and d["vs_baseline"] is None and d["config"]["workload"] == "tiny"
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1 and d["value"] > 0
     assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["e2e"]["d2h_bytes_per_step"] == 0
+
+
+def test_gpus_flag_brings_up_the_replicas_by_itself():
+    """`bench.py --gpus 2` started without a launcher (no WORLD_SIZE) spawns two ranks, which rendezvous on 127.0.0.1,
+    time the (stub) step, take the max over ranks and print ONE line with n_gpus == 2.  --dry-run keeps it off the GPU."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "20", "--warmup", "3",
+                        "--dry-run", "--backend", "gloo", "--config", "0"], capture_output=True, text=True, timeout=300, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.strip().startswith("{")]
+    assert len(lines) == 1, r.stdout
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["steps"] == 20 and d["dry_run"] is True
+    # rank 1 sleeps 2 ms per step, rank 0 1 ms: the slowest rank sets the time, both ranks' steps count
+    assert d["ms_per_step"] >= 2.0 and abs(d["value"] - 2 * 1e3 / d["ms_per_step"]) < 1e-6 * d["value"]
+
+
+def test_gpus_flag_refuses_more_ranks_than_devices():
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4096", "--steps", "1"],
+                       capture_output=True, text=True, timeout=300, env=env)
+    assert r.returncode == 2 and "CUDA device" in r.stderr

@@ -49,7 +49,8 @@ def lib() -> ctypes.CDLL:
         _lib.oracle_num_threads.restype = ctypes.c_int
         for name in ("oracle_tree_attn", "oracle_tree_attn_rows", "oracle_tree_attn_gqa", "oracle_tree_attn_rows_gqa",
                      "oracle_node_topk", "oracle_accept",
-                     "oracle_kv_compact", "oracle_check_parent", "oracle_harvest", "oracle_ancestors"):
+                     "oracle_kv_compact", "oracle_check_parent", "oracle_harvest", "oracle_ancestors", "oracle_tree_attn_n",
+                     "oracle_node_topk_n", "oracle_accept_n", "oracle_kv_compact_n"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
 
@@ -63,10 +64,16 @@ def _c(a, dt) -> np.ndarray:
     return a
 
 
-def tree_attn(q, k_cache, v_cache, row_off, ctx_len, parent, scale: float, want_lse: bool = True
+def _nn(n_nodes, S):
+    """n_nodes [S] int32 or None (every sequence has all B nodes)."""
+    return None if n_nodes is None else _c(n_nodes, np.int32).reshape(S)
+
+
+def tree_attn(q, k_cache, v_cache, row_off, ctx_len, parent, scale: float, want_lse: bool = True, n_nodes=None
               ) -> Tuple[np.ndarray, Optional[np.ndarray]]:
     """q uint16 [S][B][H][D]; caches uint16 [rows][Hkv][D] (Hkv == H: multi-head attention; Hkv a divisor of H:
     grouped-query attention, query head h reads key/value head h // (H // Hkv)).
+    n_nodes [S] (optional): nodes i >= n_nodes[s] do not exist; their output rows stay zero.
     Returns out fp64 [S][B][H][D], lse [S][B][H]."""
     q = _c(q, np.uint16); k_cache = _c(k_cache, np.uint16); v_cache = _c(v_cache, np.uint16)
     S, B, H, D = q.shape
@@ -77,10 +84,11 @@ def tree_attn(q, k_cache, v_cache, row_off, ctx_len, parent, scale: float, want_
     parent = _c(parent, np.int32).reshape(S, B)
     out = np.zeros((S, B, H, D), dtype=np.float64)
     lse = np.zeros((S, B, H), dtype=np.float64) if want_lse else None
-    rc = lib().oracle_tree_attn_gqa(_ptr(q, ctypes.c_uint16), _ptr(k_cache, ctypes.c_uint16), _ptr(v_cache, ctypes.c_uint16),
-                                    _ptr(row_off, ctypes.c_int64), _ptr(ctx_len, ctypes.c_int32), _ptr(parent, ctypes.c_int32),
-                                    ctypes.c_int(S), ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D),
-                                    ctypes.c_double(scale), _ptr(out, ctypes.c_double), _ptr(lse, ctypes.c_double))
+    nn = _nn(n_nodes, S)
+    rc = lib().oracle_tree_attn_n(_ptr(q, ctypes.c_uint16), _ptr(k_cache, ctypes.c_uint16), _ptr(v_cache, ctypes.c_uint16),
+                                  _ptr(row_off, ctypes.c_int64), _ptr(ctx_len, ctypes.c_int32), _ptr(parent, ctypes.c_int32),
+                                  _ptr(nn, ctypes.c_int32), ctypes.c_int(S), ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(Hkv),
+                                  ctypes.c_int(D), ctypes.c_double(scale), _ptr(out, ctypes.c_double), _ptr(lse, ctypes.c_double))
     if rc != 0:
         raise ValueError("oracle_tree_attn failed: rc=%d (invalid parent[]?)" % rc)
     return out, lse
@@ -111,24 +119,27 @@ def tree_attn_rows(q, k_cache, v_cache, row_off, ctx_len, parent, scale: float, 
     return out, lse
 
 
-def node_topk(logits, k: int, V: Optional[int] = None) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
-    """logits uint16 [rows][ldl] (first V columns used).  Returns argmax [rows], ids [rows][k], vals fp64 [rows][k]."""
+def node_topk(logits, k: int, V: Optional[int] = None, n_nodes=None, B: int = 0
+              ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """logits uint16 [rows][ldl] (first V columns used).  Returns argmax [rows], ids [rows][k], vals fp64 [rows][k].
+    n_nodes [rows / B] with B (optional): rows of nodes that do not exist are skipped and stay zero."""
     logits = _c(logits, np.uint16)
     rows, ldl = logits.shape
     V = ldl if V is None else V
     argmax = np.zeros(rows, dtype=np.int32)
     ids = np.zeros((rows, k), dtype=np.int32)
     vals = np.zeros((rows, k), dtype=np.float64)
-    rc = lib().oracle_node_topk(_ptr(logits, ctypes.c_uint16), ctypes.c_int(rows), ctypes.c_int(V),
-                                ctypes.c_int64(ldl), ctypes.c_int(k), _ptr(argmax, ctypes.c_int32),
-                                _ptr(ids, ctypes.c_int32), _ptr(vals, ctypes.c_double))
+    nn = None if n_nodes is None else _nn(n_nodes, rows // B)
+    rc = lib().oracle_node_topk_n(_ptr(logits, ctypes.c_uint16), ctypes.c_int(rows), ctypes.c_int(V),
+                                  ctypes.c_int64(ldl), ctypes.c_int(k), _ptr(nn, ctypes.c_int32), ctypes.c_int(B),
+                                  _ptr(argmax, ctypes.c_int32), _ptr(ids, ctypes.c_int32), _ptr(vals, ctypes.c_double))
     if rc != 0:
         raise ValueError("oracle_node_topk failed: rc=%d" % rc)
     return argmax, ids, vals
 
 
-def accept(draft_tok, parent, argmax, tag=None) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
-    """Algorithm 3 walk.  Arrays [S][B].  Returns path [S][B], accept_len [S], bonus [S]."""
+def accept(draft_tok, parent, argmax, tag=None, n_nodes=None) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """Algorithm 3 walk.  Arrays [S][B].  Returns path [S][B], accept_len [S], bonus [S].  n_nodes [S] (optional)."""
     parent = _c(parent, np.int32)
     if parent.ndim == 1:
         parent = parent[None]
@@ -139,17 +150,17 @@ def accept(draft_tok, parent, argmax, tag=None) -> Tuple[np.ndarray, np.ndarray,
     path = np.zeros((S, B), dtype=np.int32)
     alen = np.zeros(S, dtype=np.int32)
     bonus = np.zeros(S, dtype=np.int32)
-    rc = lib().oracle_accept(_ptr(draft_tok, ctypes.c_int32), _ptr(parent, ctypes.c_int32), _ptr(argmax, ctypes.c_int32),
-                             _ptr(tag_a, ctypes.c_uint8), ctypes.c_int(S), ctypes.c_int(B),
-                             _ptr(path, ctypes.c_int32), _ptr(alen, ctypes.c_int32), _ptr(bonus, ctypes.c_int32))
+    rc = lib().oracle_accept_n(_ptr(draft_tok, ctypes.c_int32), _ptr(parent, ctypes.c_int32), _ptr(argmax, ctypes.c_int32),
+                               _ptr(tag_a, ctypes.c_uint8), _ptr(_nn(n_nodes, S), ctypes.c_int32), ctypes.c_int(S), ctypes.c_int(B),
+                               _ptr(path, ctypes.c_int32), _ptr(alen, ctypes.c_int32), _ptr(bonus, ctypes.c_int32))
     if rc != 0:
         raise ValueError("oracle_accept failed: rc=%d (invalid parent[]?)" % rc)
     return path, alen, bonus
 
 
-def kv_compact(k_cache, v_cache, row_off, ctx_len, path, accept_len
+def kv_compact(k_cache, v_cache, row_off, ctx_len, path, accept_len, n_nodes=None
                ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
-    """Out-of-place compaction.  Returns (k_out, v_out, new_ctx)."""
+    """Out-of-place compaction.  Returns (k_out, v_out, new_ctx).  n_nodes [S] (optional): 0 = the sequence has left."""
     k_cache = _c(k_cache, np.uint16); v_cache = _c(v_cache, np.uint16)
     rows, H, D = k_cache.shape
     path = _c(path, np.int32)
@@ -160,9 +171,9 @@ def kv_compact(k_cache, v_cache, row_off, ctx_len, path, accept_len
     accept_len = _c(accept_len, np.int32).reshape(S)
     k_out = k_cache.copy(); v_out = v_cache.copy()
     new_ctx = np.zeros(S, dtype=np.int32)
-    rc = lib().oracle_kv_compact(_ptr(k_cache, ctypes.c_uint16), _ptr(v_cache, ctypes.c_uint16),
+    rc = lib().oracle_kv_compact_n(_ptr(k_cache, ctypes.c_uint16), _ptr(v_cache, ctypes.c_uint16),
                                  _ptr(row_off, ctypes.c_int64), _ptr(ctx_len, ctypes.c_int32),
-                                 _ptr(path, ctypes.c_int32), _ptr(accept_len, ctypes.c_int32),
+                                 _ptr(path, ctypes.c_int32), _ptr(accept_len, ctypes.c_int32), _ptr(_nn(n_nodes, S), ctypes.c_int32),
                                  ctypes.c_int(S), ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(D),
                                  _ptr(k_out, ctypes.c_uint16), _ptr(v_out, ctypes.c_uint16), _ptr(new_ctx, ctypes.c_int32))
     if rc != 0:

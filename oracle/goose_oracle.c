@@ -15,6 +15,15 @@
  *   - kv compaction:   the paper never describes it; the reading used here is "keep the
  *     accepted nodes' K/V rows, in path order, directly after the prefix".
  *
+ * Per-sequence node counts (the paper's batched prototype pads finished requests and pays for them, App.
+ * "Batch-Size Sweep"; its Discussion leaves a production batched path open): every function that takes a tree takes
+ * an optional n_nodes[S] (NULL = B nodes everywhere).  Nodes i >= n_nodes[s] do not exist: nothing of theirs is read
+ * (parent, token, query, K/V row, logits row may hold anything) and nothing is written for them; the result for the
+ * nodes that exist is BY DEFINITION the result on the tree cut to its first n_nodes[s] nodes (a tree in topological
+ * order stays a tree when cut), and n_nodes[s] = 0 is a sequence that has left the batch: no reads, no moves,
+ * accept_len 0, bonus -1, path all -1, new_ctx = ctx.  Pinned against this file's own B-node functions on explicitly
+ * cut inputs.
+ *
  * bf16 inputs arrive as uint16 bit patterns; bf16 -> double is exact.
  * No blocking, no fusion, no reordering: one output element at a time.
  * All functions are pinned by tests that do not depend on this file's own formulas.
@@ -41,6 +50,12 @@ int oracle_num_threads(void) {
 #else
     return 1;
 #endif
+}
+
+/* nodes of sequence s: n_nodes[s] when given (it must lie in [0, B]), else B; -1 = invalid */
+static int nodes_of(const int32_t* n_nodes, int s, int B) {
+    if (!n_nodes) return B;
+    return (n_nodes[s] < 0 || n_nodes[s] > B) ? -1 : n_nodes[s];
 }
 
 /* ------------------------------------------------------------------ ancestors
@@ -87,7 +102,7 @@ int oracle_check_parent(const int32_t* parent, int B) {
  * key/value heads): the H query heads are split into Hkv groups of H/Hkv consecutive heads, and every head of a
  * group reads key/value head hk = h / (H/Hkv).  Hkv == H is ordinary multi-head attention (hk = h). */
 static int attn_row(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, int64_t row0, int ctx,
-                    const int32_t* parent, int B, int H, int Hkv, int D, double scale, int i, int h,
+                    const int32_t* parent, int B /* nodes of this sequence's tree */, int H, int Hkv, int D, double scale, int i, int h,
                     const uint16_t* qrow /* q[s][i][h][:] */, double* out /* [D] */, double* lse) {
     (void)q;
     if (Hkv < 1 || H % Hkv != 0) return -3;
@@ -125,19 +140,24 @@ static int attn_row(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, i
 }
 
 /* Full output: out fp64 [S][B][H][D], lse fp64 [S][B][H] (may be NULL). Returns 0 or <0.
- * q has H heads, the caches Hkv heads (H a multiple of Hkv). */
-int oracle_tree_attn_gqa(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, const int64_t* row_off,
-                         const int32_t* ctx_len, const int32_t* parent, int S, int B, int H, int Hkv, int D,
-                         double scale, double* out, double* lse) {
+ * q has H heads, the caches Hkv heads (H a multiple of Hkv).  n_nodes [S] or NULL: rows of nodes that do not exist are
+ * left untouched. */
+int oracle_tree_attn_n(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, const int64_t* row_off,
+                       const int32_t* ctx_len, const int32_t* parent, const int32_t* n_nodes, int S, int B, int H, int Hkv,
+                       int D, double scale, double* out, double* lse) {
     int rc = 0;
     long total = (long)S * B * H;
+    for (int s = 0; s < S; ++s)
+        if (nodes_of(n_nodes, s, B) < 0) return -4;
 #pragma omp parallel for schedule(dynamic, 4)
     for (long t = 0; t < total; ++t) {
         int h = (int)(t % H);
         int i = (int)((t / H) % B);
         int s = (int)(t / ((long)H * B));
+        const int n = nodes_of(n_nodes, s, B);
+        if (i >= n) continue;                              /* the node does not exist */
         const uint16_t* qrow = q + (((size_t)s * B + i) * H + h) * D;
-        int r = attn_row(q, kc, vc, row_off[s], ctx_len[s], parent + (size_t)s * B, B, H, Hkv, D, scale, i, h, qrow,
+        int r = attn_row(q, kc, vc, row_off[s], ctx_len[s], parent + (size_t)s * B, n, H, Hkv, D, scale, i, h, qrow,
                          out + (size_t)t * D, lse ? lse + t : NULL);
         if (r != 0) {
 #pragma omp critical
@@ -145,6 +165,12 @@ int oracle_tree_attn_gqa(const uint16_t* q, const uint16_t* kc, const uint16_t* 
         }
     }
     return rc;
+}
+
+int oracle_tree_attn_gqa(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, const int64_t* row_off,
+                         const int32_t* ctx_len, const int32_t* parent, int S, int B, int H, int Hkv, int D,
+                         double scale, double* out, double* lse) {
+    return oracle_tree_attn_n(q, kc, vc, row_off, ctx_len, parent, NULL, S, B, H, Hkv, D, scale, out, lse);
 }
 
 int oracle_tree_attn(const uint16_t* q, const uint16_t* kc, const uint16_t* vc, const int64_t* row_off,
@@ -195,12 +221,19 @@ static int cmp_vi(const void* a, const void* b) {
     return (x->idx > y->idx) - (x->idx < y->idx);
 }
 
-int oracle_node_topk(const uint16_t* logits, int rows, int V, int64_t ldl, int k,
-                     int32_t* argmax, int32_t* topk_ids, double* topk_vals) {
+/* n_nodes [rows / B] or NULL: row r = s * B + i belongs to node i of sequence s; rows of nodes that do not exist are
+ * neither read nor written. */
+int oracle_node_topk_n(const uint16_t* logits, int rows, int V, int64_t ldl, int k, const int32_t* n_nodes, int B,
+                       int32_t* argmax, int32_t* topk_ids, double* topk_vals) {
     if (k < 1 || k > V) return -1;
+    if (n_nodes && (B < 1 || rows % B != 0)) return -1;
+    if (n_nodes)
+        for (int s = 0; s < rows / B; ++s)
+            if (nodes_of(n_nodes, s, B) < 0) return -4;
     int rc = 0;
 #pragma omp parallel for schedule(dynamic, 1)
     for (int r = 0; r < rows; ++r) {
+        if (n_nodes && r % B >= n_nodes[r / B]) continue;
         vi_t* a = (vi_t*)malloc(sizeof(vi_t) * (size_t)V);
         if (!a) {
 #pragma omp critical
@@ -222,33 +255,45 @@ int oracle_node_topk(const uint16_t* logits, int rows, int V, int64_t ldl, int k
     return rc;
 }
 
+int oracle_node_topk(const uint16_t* logits, int rows, int V, int64_t ldl, int k,
+                     int32_t* argmax, int32_t* topk_ids, double* topk_vals) {
+    return oracle_node_topk_n(logits, rows, V, ldl, k, NULL, 0, argmax, topk_ids, topk_vals);
+}
+
 /* ------------------------------------------------------------------ UnifiedGreedyWalk (Algorithm 3)
  * v <- root; while v has children: if a spine-tagged child's token equals argmax[v] take it;
  * else if a branch-tagged child's token equals argmax[v] take it; else stop.  bonus = argmax[v].
  * tag == NULL: no source tags; the matching child with the lowest index is taken (with distinct
  * sibling tokens at most one child can match, so the priority never changes the path).
  * path [S][B]: path[0] = 0, then the accepted nodes, then -1.  accept_len excludes the root. */
-int oracle_accept(const int32_t* draft_tok, const int32_t* parent, const int32_t* argmax,
-                  const unsigned char* tag /* [S][B], 1 = spine child; or NULL */,
-                  int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus) {
+int oracle_accept_n(const int32_t* draft_tok, const int32_t* parent, const int32_t* argmax,
+                    const unsigned char* tag /* [S][B], 1 = spine child; or NULL */, const int32_t* n_nodes /* [S] or NULL */,
+                    int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus) {
     for (int s = 0; s < S; ++s) {
         const int32_t* par = parent + (size_t)s * B;
         const int32_t* tok = draft_tok + (size_t)s * B;
         const int32_t* am = argmax + (size_t)s * B;
         int32_t* p = path + (size_t)s * B;
-        if (oracle_check_parent(par, B) != 0) return -1;
+        const int n = nodes_of(n_nodes, s, B);             /* the walk sees the first n nodes only */
+        if (n < 0) return -4;
         for (int j = 0; j < B; ++j) p[j] = -1;
+        if (n == 0) {                                      /* the sequence has left the batch */
+            accept_len[s] = 0;
+            bonus[s] = -1;
+            continue;
+        }
+        if (oracle_check_parent(par, n) != 0) return -1;
         int v = 0, len = 0;
         p[0] = 0;
         for (;;) {
             int next = -1;
             if (tag) {
-                for (int c = v + 1; c < B && next < 0; ++c)      /* priority 1: spine child */
+                for (int c = v + 1; c < n && next < 0; ++c)      /* priority 1: spine child */
                     if (par[c] == v && tag[(size_t)s * B + c] && tok[c] == am[v]) next = c;
-                for (int c = v + 1; c < B && next < 0; ++c)      /* priority 2: branch children */
+                for (int c = v + 1; c < n && next < 0; ++c)      /* priority 2: branch children */
                     if (par[c] == v && !tag[(size_t)s * B + c] && tok[c] == am[v]) next = c;
             } else {
-                for (int c = v + 1; c < B && next < 0; ++c)
+                for (int c = v + 1; c < n && next < 0; ++c)
                     if (par[c] == v && tok[c] == am[v]) next = c;
             }
             if (next < 0) break;
@@ -262,19 +307,27 @@ int oracle_accept(const int32_t* draft_tok, const int32_t* parent, const int32_t
     return 0;
 }
 
+int oracle_accept(const int32_t* draft_tok, const int32_t* parent, const int32_t* argmax,
+                  const unsigned char* tag, int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus) {
+    return oracle_accept_n(draft_tok, parent, argmax, tag, NULL, S, B, path, accept_len, bonus);
+}
+
 /* ------------------------------------------------------------------ KV compaction (out of place)
  * k_out/v_out start as copies of the caches; row ctx+j <- row ctx+path[j] of the ORIGINAL cache,
  * j = 0..accept_len.  new_ctx = ctx + 1 + accept_len.  Rows >= new_ctx are left as they were. */
-int oracle_kv_compact(const uint16_t* kc, const uint16_t* vc, const int64_t* row_off, const int32_t* ctx_len,
-                      const int32_t* path, const int32_t* accept_len, int S, int B, int H, int D,
-                      uint16_t* k_out, uint16_t* v_out, int32_t* new_ctx) {
+int oracle_kv_compact_n(const uint16_t* kc, const uint16_t* vc, const int64_t* row_off, const int32_t* ctx_len,
+                        const int32_t* path, const int32_t* accept_len, const int32_t* n_nodes /* [S] or NULL */,
+                        int S, int B, int H, int D, uint16_t* k_out, uint16_t* v_out, int32_t* new_ctx) {
     size_t row_elems = (size_t)H * D;
     for (int s = 0; s < S; ++s) {
+        const int n = nodes_of(n_nodes, s, B);
+        if (n < 0) return -4;
+        if (n == 0) { new_ctx[s] = ctx_len[s]; continue; }     /* left the batch: nothing moves, nothing is appended */
         int L = accept_len[s];
-        if (L < 0 || L >= B) return -1;
+        if (L < 0 || L >= n) return -1;
         for (int j = 0; j <= L; ++j) {
             int src = path[(size_t)s * B + j];
-            if (src < 0 || src >= B) return -1;
+            if (src < 0 || src >= n) return -1;
             size_t dst_row = (size_t)(row_off[s] + ctx_len[s] + j);
             size_t src_row = (size_t)(row_off[s] + ctx_len[s] + src);
             memcpy(k_out + dst_row * row_elems, kc + src_row * row_elems, row_elems * sizeof(uint16_t));
@@ -283,6 +336,12 @@ int oracle_kv_compact(const uint16_t* kc, const uint16_t* vc, const int64_t* row
         new_ctx[s] = ctx_len[s] + 1 + L;
     }
     return 0;
+}
+
+int oracle_kv_compact(const uint16_t* kc, const uint16_t* vc, const int64_t* row_off, const int32_t* ctx_len,
+                      const int32_t* path, const int32_t* accept_len, int S, int B, int H, int D,
+                      uint16_t* k_out, uint16_t* v_out, int32_t* new_ctx) {
+    return oracle_kv_compact_n(kc, vc, row_off, ctx_len, path, accept_len, NULL, S, B, H, D, k_out, v_out, new_ctx);
 }
 
 /* ------------------------------------------------------------------ logit harvest into the Tier-1 adjacency table

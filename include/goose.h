@@ -31,6 +31,21 @@
  * KV cache layout: bf16 [kv_rows][H][D], token-major.  Sequence s owns rows
  * row_off[s] .. row_off[s] + ctx_len[s] + B - 1: first its ctx_len[s] prefix tokens, then the
  * K/V of tree node i at row row_off[s] + ctx_len[s] + i (written by the caller before the call).
+ *
+ * Per-sequence node counts.  The paper's batched prototype keeps finished requests in the batch as
+ * padding and pays for them (App. "Batch-Size Sweep"); its Discussion leaves a production batched path
+ * open.  Every call that takes a tree takes an optional device array n_nodes int32 [S] (NULL = every tree
+ * has B nodes): sequence s has the nodes 0 .. n_nodes[s]-1 of its arrays (B stays the stride of q, out,
+ * parent, draft_tok and of the logits rows).  Nodes i >= n_nodes[s] do not exist: their parent, token,
+ * query, logits row and K/V row are never read (they may hold anything, NaN included), nothing is written
+ * for them (out, lse, argmax, topk rows keep their contents; path entries are -1), and the sequence needs
+ * only ctx_len[s] + n_nodes[s] cache rows.  The results for the nodes that exist are those of the tree
+ * cut to its first n_nodes[s] nodes.  n_nodes[s] = 0 is a sequence that has left the batch: nothing of
+ * it is read (row_off / ctx_len excepted) or moved; accept_len 0, bonus -1, path all -1,
+ * new_ctx_len = ctx_len.  A value outside [0, B] is treated as 0 and sets GOOSE_ST_BAD_NODES.
+ * The top-k then reads only the logits rows of nodes that exist (V * 2 bytes saved per absent node).
+ * Trees padded by goose_pad_tree instead (n_nodes = NULL) are verified as B-node trees: the padding nodes'
+ * K/V rows and logits rows ARE read then and must hold finite values.
  */
 #ifndef GOOSE_H_
 #define GOOSE_H_
@@ -59,6 +74,7 @@ extern "C" {
 #define GOOSE_ST_BAD_PATH     2   /* path[] / accept_len[] handed to goose_kv_compact is invalid */
 #define GOOSE_ST_TIMEOUT      4   /* a device-side wait ran out of polls */
 #define GOOSE_ST_BAD_ROWS     8   /* row_off[] / ctx_len[] put a sequence's rows outside [0, kv_rows): nothing moved */
+#define GOOSE_ST_BAD_NODES   16   /* n_nodes[s] outside [0, B]: the sequence is treated as having left the batch */
 
 /* attention kernel selection (goose_set_attn_impl) */
 #define GOOSE_ATTN_AUTO  0
@@ -88,12 +104,12 @@ int goose_set_attn_impl(goose_ctx* ctx, int impl);
  * ancestor a of i, i included.  bf16 inputs, fp32 accumulation, bf16 output (round to nearest even).
  *   q        bf16 [S][B][H][D]                       16-byte aligned
  *   k_cache, v_cache  bf16 [kv_rows][H][D]           16-byte aligned; kv_rows = rows allocated
- *   row_off  int64 [S], ctx_len int32 [S], parent int32 [S][B]   (device arrays)
+ *   row_off  int64 [S], ctx_len int32 [S], parent int32 [S][B], n_nodes int32 [S] or NULL   (device arrays)
  *   out      bf16 [S][B][H][D]; lse fp32 [S][B][H] = log-sum-exp of the scaled scores, or NULL
  * Rows row_off[s]+ctx_len[s]+B .. are never read as values (their contents may be anything).
  * ctx_len[s] = 0 is legal.  S <= max_S, B <= max_B, H <= max_H, D == 128, 0 < scale < 1e30.       */
 int goose_tree_attn(goose_ctx* ctx, const void* q, const void* k_cache, const void* v_cache, int64_t kv_rows,
-                    const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
+                    const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent, const int32_t* n_nodes,
                     int S, int B, int H, int D, float scale, void* out, float* lse, void* stream);
 
 /* Same for grouped-query attention, the head layout of the 8B models of the paper's evaluation (Sec. 5 set-up: 32
@@ -104,7 +120,7 @@ int goose_tree_attn(goose_ctx* ctx, const void* q, const void* k_cache, const vo
  * key/value rows of a head are read once per group while B * (H / Hkv) <= 128, and once per
  * ceil(B / floor(128 / (H / Hkv))) otherwise.  Other arguments, limits and errors as goose_tree_attn.          */
 int goose_tree_attn_gqa(goose_ctx* ctx, const void* q, const void* k_cache, const void* v_cache, int64_t kv_rows,
-                        const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
+                        const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent, const int32_t* n_nodes,
                         int S, int B, int H, int Hkv, int D, float scale, void* out, float* lse, void* stream);
 
 /* Per-node argmax and top-k (Algorithm 3 step 2; App. C.1 "aggressive logit harvesting": every
@@ -113,9 +129,11 @@ int goose_tree_attn_gqa(goose_ctx* ctx, const void* q, const void* k_cache, cons
  * (value descending, index ascending); -0.0 equals +0.0; argmax[r] = topk_ids[r][0].
  *   logits bf16 [rows][ldl]  16-byte aligned, ldl % 8 == 0, ldl >= V, finite values
  *   1 <= k <= min(V, GOOSE_MAX_K); V <= GOOSE_MAX_V
- *   argmax int32 [rows]; topk_ids int32 [rows][k]; topk_vals fp32 [rows][k] (exact values) or NULL */
+ *   argmax int32 [rows]; topk_ids int32 [rows][k]; topk_vals fp32 [rows][k] (exact values) or NULL
+ *   n_nodes int32 [rows / B] or NULL, with B (ignored when n_nodes is NULL; else rows % B == 0): row s * B + i
+ *   is the row of node i of sequence s and is skipped -- not read, outputs untouched -- when i >= n_nodes[s]  */
 int goose_node_topk(goose_ctx* ctx, const void* logits, int rows, int V, int64_t ldl, int k,
-                    int32_t* argmax, int32_t* topk_ids, float* topk_vals, void* stream);
+                    const int32_t* n_nodes, int B, int32_t* argmax, int32_t* topk_ids, float* topk_vals, void* stream);
 
 /* Harvest of a forward's logits into the Tier-1 (unigram) adjacency table (App. C.1 "Aggressive logit
  * harvesting"; "Dense GPU bigram adjacency table", Tier 1: two dense |V| x K tensors with the ids and the
@@ -161,24 +179,25 @@ int goose_node_topk_static(const void* logits, int rows, int V, int64_t ldl, int
 /* Greedy acceptance walk (Algorithm 3, UnifiedGreedyWalk).  From node 0, repeatedly move to the
  * child c of the current node v with draft_tok[c] == argmax[v]; stop when no child matches.
  * If sibling tokens are not distinct the matching child with the lowest index is taken.
- *   draft_tok, parent, argmax  int32 [S][B]
+ *   draft_tok, parent, argmax  int32 [S][B]; n_nodes int32 [S] or NULL
  *   path int32 [S][B]: path[s][0] = 0, then the accepted nodes in order, then -1
  *   accept_len int32 [S]: accepted draft nodes, root excluded; bonus int32 [S] = argmax at the last
  *   accepted node.  An invalid parent[] gives accept_len 0, path {0,-1,..}, bonus -1 and status.  */
-int goose_accept(goose_ctx* ctx, const int32_t* draft_tok, const int32_t* parent, const int32_t* argmax,
-                 int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus, void* stream);
+int goose_accept(goose_ctx* ctx, const int32_t* draft_tok, const int32_t* parent, const int32_t* n_nodes,
+                 const int32_t* argmax, int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus, void* stream);
 
 /* KV compaction.  The paper does not describe cache handling after acceptance; this call keeps
  * the accepted nodes' rows in path order directly after the prefix, in place:
  * row ctx_len[s]+j <- row ctx_len[s]+path[s][j] for j = 0..accept_len[s], for K and V;
  * new_ctx_len[s] = ctx_len[s] + 1 + accept_len[s].  Rows >= new_ctx_len[s] are unspecified after
- * the call.  path must be increasing (as goose_accept produces it).
+ * the call.  path must be increasing (as goose_accept produces it).  n_nodes int32 [S] or NULL: a
+ * sequence with n_nodes[s] = 0 has left the batch (nothing moves, new_ctx_len[s] = ctx_len[s]).
  * new_ctx_len must not overlap ctx_len (GOOSE_EINVAL): every thread block of the launch reads ctx_len[s]
  * while one of them writes new_ctx_len[s].  To chain steps without a host round trip, alternate two
  * arrays: step t+1 takes step t's new_ctx_len as its ctx_len and writes the other array.             */
 int goose_kv_compact(goose_ctx* ctx, void* k_cache, void* v_cache, int64_t kv_rows,
                      const int64_t* row_off, const int32_t* ctx_len, const int32_t* path,
-                     const int32_t* accept_len, int S, int B, int H, int D,
+                     const int32_t* accept_len, const int32_t* n_nodes, int S, int B, int H, int D,
                      int32_t* new_ctx_len, void* stream);
 
 /* The whole step on one stream, in data-flow order: tree attention, node top-k (rows = S*B),
@@ -189,7 +208,7 @@ int goose_kv_compact(goose_ctx* ctx, void* k_cache, void* v_cache, int64_t kv_ro
  * ahead of their stream-order dependency on the step's earlier kernels.                              */
 int goose_verify_step(goose_ctx* ctx, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
                       const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
-                      const int32_t* draft_tok, const void* logits, int64_t ldl,
+                      const int32_t* n_nodes, const int32_t* draft_tok, const void* logits, int64_t ldl,
                       int S, int B, int H, int D, int V, int k, float scale,
                       void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
                       int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
@@ -199,7 +218,7 @@ int goose_verify_step(goose_ctx* ctx, const void* q, void* k_cache, void* v_cach
  * over the caches' Hkv heads; everything else as goose_verify_step (which is this call with Hkv == H).       */
 int goose_verify_step_gqa(goose_ctx* ctx, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
                           const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
-                          const int32_t* draft_tok, const void* logits, int64_t ldl,
+                          const int32_t* n_nodes, const int32_t* draft_tok, const void* logits, int64_t ldl,
                           int S, int B, int H, int Hkv, int D, int V, int k, float scale,
                           void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
                           int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
@@ -213,7 +232,7 @@ int goose_verify_step_gqa(goose_ctx* ctx, const void* q, void* k_cache, void* v_
  * With row_lse, adj_ids and adj_scores all NULL (table_rows ignored) this is goose_verify_step_gqa.             */
 int goose_verify_step_harvest(goose_ctx* ctx, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
                               const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
-                              const int32_t* draft_tok, const void* logits, int64_t ldl,
+                              const int32_t* n_nodes, const int32_t* draft_tok, const void* logits, int64_t ldl,
                               int S, int B, int H, int Hkv, int D, int V, int k, float scale,
                               void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
                               int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
@@ -224,7 +243,10 @@ int goose_verify_step_harvest(goose_ctx* ctx, const void* q, void* k_cache, void
  * step consumes or produces is in HOST memory (pinned memory makes the copies asynchronous):
  *   in : h_q bf16 [S][B][H][D]; h_k_new, h_v_new bf16 [S][B][H][D] = the tree nodes' K/V rows,
  *        copied to rows row_off[s]+ctx_len[s]+i; h_row_off int64 [S]; h_ctx_len int32 [S];
- *        h_parent, h_draft_tok int32 [S][B]; h_logits bf16 [S*B][V] (dense, ldl = V)
+ *        h_parent, h_draft_tok int32 [S][B]; h_n_nodes int32 [S] or NULL (validated on the host: outside
+ *        [0, B] is GOOSE_EINVAL; only the K/V rows of nodes that exist are copied; the output arrays are
+ *        copied back whole, so the output rows of nodes that do not exist are unspecified here);
+ *        h_logits bf16 [S*B][V] (dense, ldl = V)
  *   out: h_out bf16 [S][B][H][D]; h_argmax [S*B]; h_topk_ids [S*B][k]; h_topk_vals [S*B][k] or NULL;
  *        h_path [S][B]; h_accept_len, h_bonus, h_new_ctx_len [S]
  * Copies in, runs goose_verify_step, copies out, and synchronises `stream` before returning.
@@ -235,7 +257,7 @@ int goose_verify_step_harvest(goose_ctx* ctx, const void* q, void* k_cache, void
 int goose_verify_step_host(goose_ctx* ctx, void* k_cache, void* v_cache, int64_t kv_rows,
                            const void* h_q, const void* h_k_new, const void* h_v_new,
                            const int64_t* h_row_off, const int32_t* h_ctx_len,
-                           const int32_t* h_parent, const int32_t* h_draft_tok, const void* h_logits,
+                           const int32_t* h_parent, const int32_t* h_n_nodes, const int32_t* h_draft_tok, const void* h_logits,
                            int S, int B, int H, int D, int V, int k, float scale,
                            void* h_out, int32_t* h_argmax, int32_t* h_topk_ids, float* h_topk_vals,
                            int32_t* h_path, int32_t* h_accept_len, int32_t* h_bonus,
@@ -246,8 +268,8 @@ int goose_verify_step_host(goose_ctx* ctx, void* k_cache, void* v_cache, int64_t
 int goose_verify_step_host_gqa(goose_ctx* ctx, void* k_cache, void* v_cache, int64_t kv_rows,
                                const void* h_q, const void* h_k_new, const void* h_v_new,
                                const int64_t* h_row_off, const int32_t* h_ctx_len,
-                               const int32_t* h_parent, const int32_t* h_draft_tok, const void* h_logits,
-                               int S, int B, int H, int Hkv, int D, int V, int k, float scale,
+                               const int32_t* h_parent, const int32_t* h_n_nodes, const int32_t* h_draft_tok,
+                               const void* h_logits, int S, int B, int H, int Hkv, int D, int V, int k, float scale,
                                void* h_out, int32_t* h_argmax, int32_t* h_topk_ids, float* h_topk_vals,
                                int32_t* h_path, int32_t* h_accept_len, int32_t* h_bonus,
                                int32_t* h_new_ctx_len, void* stream);
@@ -267,7 +289,10 @@ int goose_build_spine_tree(int32_t anchor, const int32_t* chain, int m, const in
                            int32_t* n_nodes, int32_t* n_spine);
 
 /* Fill nodes n_nodes..B-1 with padding (children of the root with negative tokens, which no argmax can match), so
- * that a tree with fewer than B nodes can be verified by kernels that take a fixed B.                           */
+ * that a tree with fewer than B nodes can be verified as a B-node tree (n_nodes = NULL in the calls above).  The
+ * padding nodes' K/V rows and logits rows are then read like any other node's and must hold finite values (a
+ * padding key gets weight 0 in the softmax of every real node, and 0 x NaN is NaN).  Passing the node count in
+ * n_nodes[] instead needs no padding, reads none of those rows and leaves no such requirement.                  */
 int goose_pad_tree(int32_t* draft_tok, int32_t* parent, int n_nodes, int B);
 
 /* ContextMatch (paragraph after Algorithm 2): n-gram lookup with n in {5, 4, 3} of the last n tokens of ctx at

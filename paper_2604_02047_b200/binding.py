@@ -26,7 +26,7 @@ EXPORTS = [
 ]
 
 ATTN_AUTO, ATTN_MMA, ATTN_UMMA = 0, 1, 2
-ST_BAD_PARENT, ST_BAD_PATH, ST_TIMEOUT, ST_BAD_ROWS = 1, 2, 4, 8
+ST_BAD_PARENT, ST_BAD_PATH, ST_TIMEOUT, ST_BAD_ROWS, ST_BAD_NODES = 1, 2, 4, 8, 16
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -77,6 +77,24 @@ def _dev(t: torch.Tensor, dtype: torch.dtype, name: str) -> torch.Tensor:
     if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
         raise GooseError("%s must be a contiguous CUDA tensor of dtype %s" % (name, dtype))
     return t
+
+
+def _nn(n_nodes: Optional[torch.Tensor], S: int) -> Optional[torch.Tensor]:
+    """Per-sequence node counts: a contiguous int32 CUDA tensor [S], or None (every tree has all B nodes)."""
+    if n_nodes is None:
+        return None
+    _dev(n_nodes, torch.int32, "n_nodes")
+    if n_nodes.numel() != S:
+        raise GooseError("n_nodes must have one entry per sequence")
+    return n_nodes
+
+
+def _host_nn(h_n_nodes: Optional[torch.Tensor], S: int) -> Optional[torch.Tensor]:
+    if h_n_nodes is None:
+        return None
+    if h_n_nodes.is_cuda or h_n_nodes.dtype != torch.int32 or not h_n_nodes.is_contiguous() or h_n_nodes.numel() != S:
+        raise GooseError("h_n_nodes must be a contiguous int32 host tensor [S]")
+    return h_n_nodes
 
 
 def _kv_heads(k_cache: torch.Tensor, v_cache: torch.Tensor) -> int:
@@ -140,7 +158,8 @@ class Goose:
     # ------------------------------------------------------------------ the four calls
     def tree_attn(self, q, k_cache, v_cache, row_off, ctx_len, parent, scale: float,
                   out: Optional[torch.Tensor] = None, want_lse: bool = False,
-                  lse: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, Optional[torch.Tensor]]:
+                  lse: Optional[torch.Tensor] = None, n_nodes: Optional[torch.Tensor] = None
+                  ) -> Tuple[torch.Tensor, Optional[torch.Tensor]]:
         _dev(q, torch.bfloat16, "q"); _dev(k_cache, torch.bfloat16, "k_cache"); _dev(v_cache, torch.bfloat16, "v_cache")
         _dev(row_off, torch.int64, "row_off"); _dev(ctx_len, torch.int32, "ctx_len"); _dev(parent, torch.int32, "parent")
         S, B, H, D = q.shape
@@ -150,14 +169,15 @@ class Goose:
         if want_lse and lse is None:
             lse = torch.empty((S, B, H), dtype=torch.float32, device=q.device)
         _check(self.lib.goose_tree_attn(self.h, _p(q), _p(k_cache), _p(v_cache), ctypes.c_int64(k_cache.shape[0]),
-                                        _p(row_off), _p(ctx_len), _p(parent), ctypes.c_int(S), ctypes.c_int(B),
+                                        _p(row_off), _p(ctx_len), _p(parent), _p(_nn(n_nodes, S)), ctypes.c_int(S), ctypes.c_int(B),
                                         ctypes.c_int(H), ctypes.c_int(D), ctypes.c_float(scale), _p(out), _p(lse),
                                         _stream()), "goose_tree_attn")
         return out, lse
 
     def tree_attn_gqa(self, q, k_cache, v_cache, row_off, ctx_len, parent, scale: float,
                       out: Optional[torch.Tensor] = None, want_lse: bool = False,
-                      lse: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, Optional[torch.Tensor]]:
+                      lse: Optional[torch.Tensor] = None, n_nodes: Optional[torch.Tensor] = None
+                      ) -> Tuple[torch.Tensor, Optional[torch.Tensor]]:
         """Grouped-query attention: q [S][B][H][D], caches [rows][Hkv][D]; Hkv is read from the caches' shape."""
         _dev(q, torch.bfloat16, "q"); _dev(k_cache, torch.bfloat16, "k_cache"); _dev(v_cache, torch.bfloat16, "v_cache")
         _dev(row_off, torch.int64, "row_off"); _dev(ctx_len, torch.int32, "ctx_len"); _dev(parent, torch.int32, "parent")
@@ -168,20 +188,28 @@ class Goose:
         if want_lse and lse is None:
             lse = torch.empty((S, B, H), dtype=torch.float32, device=q.device)
         _check(self.lib.goose_tree_attn_gqa(self.h, _p(q), _p(k_cache), _p(v_cache), ctypes.c_int64(k_cache.shape[0]),
-                                            _p(row_off), _p(ctx_len), _p(parent), ctypes.c_int(S), ctypes.c_int(B),
+                                            _p(row_off), _p(ctx_len), _p(parent), _p(_nn(n_nodes, S)), ctypes.c_int(S), ctypes.c_int(B),
                                             ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D), ctypes.c_float(scale),
                                             _p(out), _p(lse), _stream()), "goose_tree_attn_gqa")
         return out, lse
 
-    def node_topk(self, logits, k: int, V: Optional[int] = None, want_vals: bool = True):
+    def node_topk(self, logits, k: int, V: Optional[int] = None, want_vals: bool = True,
+                  n_nodes: Optional[torch.Tensor] = None, B: int = 0, outs=None):
+        """``n_nodes`` [rows / B] with ``B``: rows of nodes that do not exist are skipped (not read, outputs untouched;
+        pass ``outs`` = (argmax, ids, vals) to see what they held before)."""
         _dev(logits, torch.bfloat16, "logits")
         rows, ldl = logits.shape
         V = ldl if V is None else V
-        argmax = torch.empty(rows, dtype=torch.int32, device=logits.device)
-        ids = torch.empty((rows, k), dtype=torch.int32, device=logits.device)
-        vals = torch.empty((rows, k), dtype=torch.float32, device=logits.device) if want_vals else None
+        if outs is not None:
+            argmax, ids, vals = outs
+        else:
+            argmax = torch.empty(rows, dtype=torch.int32, device=logits.device)
+            ids = torch.empty((rows, k), dtype=torch.int32, device=logits.device)
+            vals = torch.empty((rows, k), dtype=torch.float32, device=logits.device) if want_vals else None
+        nn = None if n_nodes is None else _nn(n_nodes, rows // max(B, 1))
         _check(self.lib.goose_node_topk(self.h, _p(logits), ctypes.c_int(rows), ctypes.c_int(V), ctypes.c_int64(ldl),
-                                        ctypes.c_int(k), _p(argmax), _p(ids), _p(vals), _stream()), "goose_node_topk")
+                                        ctypes.c_int(k), _p(nn), ctypes.c_int(B), _p(argmax), _p(ids), _p(vals), _stream()),
+               "goose_node_topk")
         return argmax, ids, vals
 
     def harvest(self, logits, k: int, row_tok, adj_ids, adj_scores, V: Optional[int] = None):
@@ -201,24 +229,24 @@ class Goose:
                "goose_harvest")
         return argmax, ids, vals, lse
 
-    def accept(self, draft_tok, parent, argmax):
+    def accept(self, draft_tok, parent, argmax, n_nodes: Optional[torch.Tensor] = None):
         _dev(draft_tok, torch.int32, "draft_tok"); _dev(parent, torch.int32, "parent"); _dev(argmax, torch.int32, "argmax")
         S, B = parent.shape
         path = torch.empty((S, B), dtype=torch.int32, device=parent.device)
         alen = torch.empty(S, dtype=torch.int32, device=parent.device)
         bonus = torch.empty(S, dtype=torch.int32, device=parent.device)
-        _check(self.lib.goose_accept(self.h, _p(draft_tok), _p(parent), _p(argmax), ctypes.c_int(S), ctypes.c_int(B),
+        _check(self.lib.goose_accept(self.h, _p(draft_tok), _p(parent), _p(_nn(n_nodes, S)), _p(argmax), ctypes.c_int(S), ctypes.c_int(B),
                                      _p(path), _p(alen), _p(bonus), _stream()), "goose_accept")
         return path, alen, bonus
 
-    def kv_compact(self, k_cache, v_cache, row_off, ctx_len, path, accept_len):
+    def kv_compact(self, k_cache, v_cache, row_off, ctx_len, path, accept_len, n_nodes: Optional[torch.Tensor] = None):
         _dev(k_cache, torch.bfloat16, "k_cache"); _dev(v_cache, torch.bfloat16, "v_cache")
         _dev(path, torch.int32, "path"); _dev(accept_len, torch.int32, "accept_len")
         rows, H, D = k_cache.shape
         S, B = path.shape
         new_ctx = torch.empty(S, dtype=torch.int32, device=path.device)
         _check(self.lib.goose_kv_compact(self.h, _p(k_cache), _p(v_cache), ctypes.c_int64(rows), _p(row_off),
-                                         _p(ctx_len), _p(path), _p(accept_len), ctypes.c_int(S), ctypes.c_int(B),
+                                         _p(ctx_len), _p(path), _p(accept_len), _p(_nn(n_nodes, S)), ctypes.c_int(S), ctypes.c_int(B),
                                          ctypes.c_int(H), ctypes.c_int(D), _p(new_ctx), _stream()), "goose_kv_compact")
         return new_ctx
 
@@ -237,7 +265,7 @@ class Goose:
         )
 
     def verify_step(self, q, k_cache, v_cache, row_off, ctx_len, parent, draft_tok, logits, k: int, scale: float,
-                    outs: Optional[dict] = None, V: Optional[int] = None) -> dict:
+                    outs: Optional[dict] = None, V: Optional[int] = None, n_nodes: Optional[torch.Tensor] = None) -> dict:
         S, B, H, D = q.shape
         _same_heads(k_cache, v_cache, H, "verify_step")
         ldl = logits.shape[1]
@@ -246,7 +274,7 @@ class Goose:
             outs = self.alloc_step_outputs(S, B, H, D, k, q.device)
         _check(self.lib.goose_verify_step(
             self.h, _p(q), _p(k_cache), _p(v_cache), ctypes.c_int64(k_cache.shape[0]), _p(row_off), _p(ctx_len),
-            _p(parent), _p(draft_tok), _p(logits), ctypes.c_int64(ldl), ctypes.c_int(S), ctypes.c_int(B),
+            _p(parent), _p(_nn(n_nodes, S)), _p(draft_tok), _p(logits), ctypes.c_int64(ldl), ctypes.c_int(S), ctypes.c_int(B),
             ctypes.c_int(H), ctypes.c_int(D), ctypes.c_int(V), ctypes.c_int(k), ctypes.c_float(scale),
             _p(outs["out"]), _p(outs.get("lse")), _p(outs["argmax"]), _p(outs["topk_ids"]), _p(outs["topk_vals"]),
             _p(outs["path"]), _p(outs["accept_len"]), _p(outs["bonus"]), _p(outs["new_ctx_len"]), _stream()),
@@ -254,7 +282,7 @@ class Goose:
         return outs
 
     def verify_step_gqa(self, q, k_cache, v_cache, row_off, ctx_len, parent, draft_tok, logits, k: int, scale: float,
-                        outs: Optional[dict] = None, V: Optional[int] = None) -> dict:
+                        outs: Optional[dict] = None, V: Optional[int] = None, n_nodes: Optional[torch.Tensor] = None) -> dict:
         """The whole step with grouped-query attention (Hkv is read from the caches' shape)."""
         S, B, H, D = q.shape
         Hkv = _kv_heads(k_cache, v_cache)
@@ -264,7 +292,7 @@ class Goose:
             outs = self.alloc_step_outputs(S, B, H, D, k, q.device)
         _check(self.lib.goose_verify_step_gqa(
             self.h, _p(q), _p(k_cache), _p(v_cache), ctypes.c_int64(k_cache.shape[0]), _p(row_off), _p(ctx_len),
-            _p(parent), _p(draft_tok), _p(logits), ctypes.c_int64(ldl), ctypes.c_int(S), ctypes.c_int(B),
+            _p(parent), _p(_nn(n_nodes, S)), _p(draft_tok), _p(logits), ctypes.c_int64(ldl), ctypes.c_int(S), ctypes.c_int(B),
             ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D), ctypes.c_int(V), ctypes.c_int(k), ctypes.c_float(scale),
             _p(outs["out"]), _p(outs.get("lse")), _p(outs["argmax"]), _p(outs["topk_ids"]), _p(outs["topk_vals"]),
             _p(outs["path"]), _p(outs["accept_len"]), _p(outs["bonus"]), _p(outs["new_ctx_len"]), _stream()),
@@ -272,7 +300,8 @@ class Goose:
         return outs
 
     def verify_step_harvest(self, q, k_cache, v_cache, row_off, ctx_len, parent, draft_tok, logits, k: int, scale: float,
-                            adj_ids, adj_scores, outs: Optional[dict] = None, V: Optional[int] = None) -> dict:
+                            adj_ids, adj_scores, outs: Optional[dict] = None, V: Optional[int] = None,
+                            n_nodes: Optional[torch.Tensor] = None) -> dict:
         """The whole step plus the harvest of its logits into the adjacency table (updated in place); multi-head or
         grouped-query (Hkv is read from the caches' shape).  ``outs`` gains ``row_lse`` [S*B]."""
         S, B, H, D = q.shape
@@ -286,7 +315,7 @@ class Goose:
             outs["row_lse"] = torch.empty(S * B, dtype=torch.float32, device=q.device)
         _check(self.lib.goose_verify_step_harvest(
             self.h, _p(q), _p(k_cache), _p(v_cache), ctypes.c_int64(k_cache.shape[0]), _p(row_off), _p(ctx_len),
-            _p(parent), _p(draft_tok), _p(logits), ctypes.c_int64(ldl), ctypes.c_int(S), ctypes.c_int(B),
+            _p(parent), _p(_nn(n_nodes, S)), _p(draft_tok), _p(logits), ctypes.c_int64(ldl), ctypes.c_int(S), ctypes.c_int(B),
             ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D), ctypes.c_int(V), ctypes.c_int(k), ctypes.c_float(scale),
             _p(outs["out"]), _p(outs.get("lse")), _p(outs["argmax"]), _p(outs["topk_ids"]), _p(outs["topk_vals"]),
             _p(outs["path"]), _p(outs["accept_len"]), _p(outs["bonus"]), _p(outs["new_ctx_len"]), _p(outs["row_lse"]),
@@ -294,7 +323,8 @@ class Goose:
         return outs
 
     def verify_step_host_gqa(self, k_cache, v_cache, h_q, h_k_new, h_v_new, h_row_off, h_ctx_len, h_parent,
-                             h_draft_tok, h_logits, k: int, scale: float, h_outs: dict) -> dict:
+                             h_draft_tok, h_logits, k: int, scale: float, h_outs: dict,
+                             h_n_nodes: Optional[torch.Tensor] = None) -> dict:
         """End-to-end call with grouped-query attention: h_k_new / h_v_new are [S][B][Hkv][D]."""
         S, B, H, D = h_q.shape
         Hkv = _kv_heads(k_cache, v_cache)
@@ -306,7 +336,7 @@ class Goose:
             raise GooseError("h_k_new / h_v_new must be [S][B][Hkv][D]")
         _check(self.lib.goose_verify_step_host_gqa(
             self.h, _p(k_cache), _p(v_cache), ctypes.c_int64(k_cache.shape[0]), _p(h_q), _p(h_k_new), _p(h_v_new),
-            _p(h_row_off), _p(h_ctx_len), _p(h_parent), _p(h_draft_tok), _p(h_logits), ctypes.c_int(S),
+            _p(h_row_off), _p(h_ctx_len), _p(h_parent), _p(_host_nn(h_n_nodes, S)), _p(h_draft_tok), _p(h_logits), ctypes.c_int(S),
             ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(Hkv), ctypes.c_int(D), ctypes.c_int(V), ctypes.c_int(k),
             ctypes.c_float(scale), _p(h_outs["out"]), _p(h_outs["argmax"]), _p(h_outs["topk_ids"]),
             _p(h_outs["topk_vals"]), _p(h_outs["path"]), _p(h_outs["accept_len"]), _p(h_outs["bonus"]),
@@ -314,7 +344,8 @@ class Goose:
         return h_outs
 
     def verify_step_host(self, k_cache, v_cache, h_q, h_k_new, h_v_new, h_row_off, h_ctx_len, h_parent,
-                         h_draft_tok, h_logits, k: int, scale: float, h_outs: dict) -> dict:
+                         h_draft_tok, h_logits, k: int, scale: float, h_outs: dict,
+                         h_n_nodes: Optional[torch.Tensor] = None) -> dict:
         """End-to-end call: per-step inputs and outputs are (pinned) host tensors; the prefix KV cache
         is device state.  Synchronises the current stream before returning."""
         S, B, H, D = h_q.shape
@@ -325,7 +356,7 @@ class Goose:
                 raise GooseError("verify_step_host takes contiguous host tensors")
         _check(self.lib.goose_verify_step_host(
             self.h, _p(k_cache), _p(v_cache), ctypes.c_int64(k_cache.shape[0]), _p(h_q), _p(h_k_new), _p(h_v_new),
-            _p(h_row_off), _p(h_ctx_len), _p(h_parent), _p(h_draft_tok), _p(h_logits), ctypes.c_int(S),
+            _p(h_row_off), _p(h_ctx_len), _p(h_parent), _p(_host_nn(h_n_nodes, S)), _p(h_draft_tok), _p(h_logits), ctypes.c_int(S),
             ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(D), ctypes.c_int(V), ctypes.c_int(k),
             ctypes.c_float(scale), _p(h_outs["out"]), _p(h_outs["argmax"]), _p(h_outs["topk_ids"]),
             _p(h_outs["topk_vals"]), _p(h_outs["path"]), _p(h_outs["accept_len"]), _p(h_outs["bonus"]),

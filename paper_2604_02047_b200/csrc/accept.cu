@@ -11,7 +11,7 @@ namespace goose {
 
 __global__ void __launch_bounds__(32)
 accept_kernel(const int32_t* __restrict__ draft_tok, const int32_t* __restrict__ parent,
-              const int32_t* __restrict__ argmax, int B, int32_t* __restrict__ path,
+              const int32_t* __restrict__ n_nodes, const int32_t* __restrict__ argmax, int B, int32_t* __restrict__ path,
               int32_t* __restrict__ accept_len, int32_t* __restrict__ bonus, int32_t* __restrict__ status) {
     const int s = blockIdx.x, lane = threadIdx.x;
     const int32_t* par = parent + (size_t)s * B;
@@ -20,6 +20,17 @@ accept_kernel(const int32_t* __restrict__ draft_tok, const int32_t* __restrict__
     int32_t* p = path + (size_t)s * B;
     pdl_wait();
     pdl_trigger();
+    // the walk sees the first nn nodes of the tree; nn = 0: the sequence has left the batch (nothing of it is read)
+    const int nn = nodes_of(n_nodes, s, B);
+    if (nn == 0) {
+        for (int c = lane; c < B; c += 32) p[c] = -1;
+        if (lane == 0) {
+            accept_len[s] = 0;
+            bonus[s] = -1;
+            if (nodes_bad(n_nodes, s, B)) atomicOr(&status[s], GOOSE_ST_BAD_NODES);
+        }
+        return;
+    }
 
     constexpr int kPer = kMaxB / 32;
     int my_par[kPer];
@@ -30,7 +41,7 @@ accept_kernel(const int32_t* __restrict__ draft_tok, const int32_t* __restrict__
         int c = lane + 32 * t;
         my_par[t] = -2;
         my_match[t] = false;
-        if (c < B) {
+        if (c < nn) {
             int pp = par[c];
             my_par[t] = pp;
             if (c == 0) bad |= (pp != -1);
@@ -50,11 +61,11 @@ accept_kernel(const int32_t* __restrict__ draft_tok, const int32_t* __restrict__
 #pragma unroll
     for (int t = 0; t < kPer; ++t) {
         int c = lane + 32 * t;
-        if (c >= 1 && c < B) my_match[t] = (tok[c] == am[my_par[t]]);
+        if (c >= 1 && c < nn) my_match[t] = (tok[c] == am[my_par[t]]);
     }
     __syncwarp();
     int v = 0, len = 0;
-    for (int step = 0; step < B - 1; ++step) {
+    for (int step = 0; step < nn - 1; ++step) {
         int cand = 0x7FFFFFFF;
 #pragma unroll
         for (int t = kPer - 1; t >= 0; --t)
@@ -71,10 +82,11 @@ accept_kernel(const int32_t* __restrict__ draft_tok, const int32_t* __restrict__
     }
 }
 
-cudaError_t launch_accept(goose_ctx* c, const int32_t* draft_tok, const int32_t* parent, const int32_t* argmax,
-                          int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus, cudaStream_t st) {
+cudaError_t launch_accept(goose_ctx* c, const int32_t* draft_tok, const int32_t* parent, const int32_t* n_nodes,
+                          const int32_t* argmax, int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus,
+                          cudaStream_t st) {
     if (S == 0) return cudaSuccess;
-    cudaError_t e = launch_pdl(accept_kernel, dim3(S), dim3(32), 0, st, draft_tok, parent, argmax, B, path,
+    cudaError_t e = launch_pdl(accept_kernel, dim3(S), dim3(32), 0, st, draft_tok, parent, n_nodes, argmax, B, path,
                                accept_len, bonus, c->status);
     c->launches++;
     return e;

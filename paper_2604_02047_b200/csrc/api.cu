@@ -149,14 +149,14 @@ int goose_set_attn_impl(goose_ctx* c, int impl) {
 int64_t goose_launch_count(goose_ctx* c) { return c ? c->launches : -1; }
 
 int goose_tree_attn(goose_ctx* c, const void* q, const void* k_cache, const void* v_cache, int64_t kv_rows,
-                    const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
+                    const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent, const int32_t* n_nodes,
                     int S, int B, int H, int D, float scale, void* out, float* lse, void* stream) {
-    return goose_tree_attn_gqa(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, S, B, H, H, D, scale, out, lse,
-                               stream);
+    return goose_tree_attn_gqa(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, n_nodes, S, B, H, H, D, scale, out,
+                               lse, stream);
 }
 
 int goose_tree_attn_gqa(goose_ctx* c, const void* q, const void* k_cache, const void* v_cache, int64_t kv_rows,
-                        const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
+                        const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent, const int32_t* n_nodes,
                         int S, int B, int H, int Hkv, int D, float scale, void* out, float* lse, void* stream) {
     int rc = check_shape(c, S, B, H, D);
     if (rc) return rc;
@@ -172,24 +172,25 @@ int goose_tree_attn_gqa(goose_ctx* c, const void* q, const void* k_cache, const 
     cudaError_t e;
     if (impl == GOOSE_ATTN_UMMA)
         e = goose::launch_tree_attn_umma(c, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_cache,
-                                         (const __nv_bfloat16*)v_cache, kv_rows, row_off, ctx_len, parent, S, B, H, Hkv,
-                                         scale, (__nv_bfloat16*)out, lse, st);
+                                         (const __nv_bfloat16*)v_cache, kv_rows, row_off, ctx_len, parent, n_nodes, S, B, H,
+                                         Hkv, scale, (__nv_bfloat16*)out, lse, st);
     else
         e = goose::launch_tree_attn_mma(c, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_cache,
-                                        (const __nv_bfloat16*)v_cache, kv_rows, row_off, ctx_len, parent, S, B, H, Hkv,
-                                        scale, (__nv_bfloat16*)out, lse, st);
+                                        (const __nv_bfloat16*)v_cache, kv_rows, row_off, ctx_len, parent, n_nodes, S, B, H,
+                                        Hkv, scale, (__nv_bfloat16*)out, lse, st);
     if (e != cudaSuccess) return cuda_fail(e);
     return GOOSE_OK;
 }
 
 int goose_node_topk(goose_ctx* c, const void* logits, int rows, int V, int64_t ldl, int k,
-                    int32_t* argmax, int32_t* topk_ids, float* topk_vals, void* stream) {
+                    const int32_t* n_nodes, int B, int32_t* argmax, int32_t* topk_ids, float* topk_vals, void* stream) {
     if (!c || !on_ctx_device(c) || !logits || !argmax || !topk_ids) return GOOSE_EINVAL;
     if (rows < 0 || rows > c->topk_rows_cap) return GOOSE_EINVAL;
+    if (n_nodes && (B < 1 || B > GOOSE_MAX_B || rows % B != 0)) return GOOSE_EINVAL;
     if (V < 1 || V > GOOSE_MAX_V || ldl < V || (ldl & 7) != 0 || !aligned16(logits)) return GOOSE_EINVAL;
     if (k < 1 || k > GOOSE_MAX_K || k > V) return GOOSE_EINVAL;
     cudaError_t e = goose::launch_node_topk(c, (const __nv_bfloat16*)logits, rows, V, ldl, k, argmax, topk_ids,
-                                            topk_vals, nullptr, static_cast<cudaStream_t>(stream));
+                                            topk_vals, nullptr, static_cast<cudaStream_t>(stream), false, n_nodes, B);
     if (e != cudaSuccess) return cuda_fail(e);
     return GOOSE_OK;
 }
@@ -213,11 +214,11 @@ int goose_harvest(goose_ctx* c, const void* logits, int rows, int V, int64_t ldl
     return GOOSE_OK;
 }
 
-int goose_accept(goose_ctx* c, const int32_t* draft_tok, const int32_t* parent, const int32_t* argmax,
-                 int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus, void* stream) {
+int goose_accept(goose_ctx* c, const int32_t* draft_tok, const int32_t* parent, const int32_t* n_nodes,
+                 const int32_t* argmax, int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus, void* stream) {
     if (!c || !on_ctx_device(c) || !draft_tok || !parent || !argmax || !path || !accept_len || !bonus) return GOOSE_EINVAL;
     if (S < 0 || S > c->max_S || B < 1 || B > c->max_B) return GOOSE_EINVAL;
-    cudaError_t e = goose::launch_accept(c, draft_tok, parent, argmax, S, B, path, accept_len, bonus,
+    cudaError_t e = goose::launch_accept(c, draft_tok, parent, n_nodes, argmax, S, B, path, accept_len, bonus,
                                          static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(e);
     return GOOSE_OK;
@@ -225,7 +226,7 @@ int goose_accept(goose_ctx* c, const int32_t* draft_tok, const int32_t* parent, 
 
 int goose_kv_compact(goose_ctx* c, void* k_cache, void* v_cache, int64_t kv_rows,
                      const int64_t* row_off, const int32_t* ctx_len, const int32_t* path,
-                     const int32_t* accept_len, int S, int B, int H, int D,
+                     const int32_t* accept_len, const int32_t* n_nodes, int S, int B, int H, int D,
                      int32_t* new_ctx_len, void* stream) {
     int rc = check_shape(c, S, B, H, D);
     if (rc) return rc;
@@ -233,7 +234,7 @@ int goose_kv_compact(goose_ctx* c, void* k_cache, void* v_cache, int64_t kv_rows
     if (!aligned16(k_cache) || !aligned16(v_cache) || kv_rows < 1) return GOOSE_EINVAL;
     if (ctx_arrays_overlap(ctx_len, new_ctx_len, S)) return GOOSE_EINVAL;
     cudaError_t e = goose::launch_kv_compact(c, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, row_off, ctx_len,
-                                             path, accept_len, S, B, H, kv_rows, new_ctx_len,
+                                             path, accept_len, n_nodes, S, B, H, kv_rows, new_ctx_len,
                                              static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(e);
     return GOOSE_OK;
@@ -241,25 +242,25 @@ int goose_kv_compact(goose_ctx* c, void* k_cache, void* v_cache, int64_t kv_rows
 
 int goose_verify_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
                       const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
-                      const int32_t* draft_tok, const void* logits, int64_t ldl,
+                      const int32_t* n_nodes, const int32_t* draft_tok, const void* logits, int64_t ldl,
                       int S, int B, int H, int D, int V, int k, float scale,
                       void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
                       int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
                       void* stream) {
-    return goose_verify_step_gqa(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, draft_tok, logits, ldl, S, B,
-                                 H, H, D, V, k, scale, out, lse, argmax, topk_ids, topk_vals, path, accept_len, bonus,
+    return goose_verify_step_gqa(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, n_nodes, draft_tok, logits, ldl,
+                                 S, B, H, H, D, V, k, scale, out, lse, argmax, topk_ids, topk_vals, path, accept_len, bonus,
                                  new_ctx_len, stream);
 }
 
 int goose_verify_step_gqa(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
                           const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
-                          const int32_t* draft_tok, const void* logits, int64_t ldl,
+                          const int32_t* n_nodes, const int32_t* draft_tok, const void* logits, int64_t ldl,
                           int S, int B, int H, int Hkv, int D, int V, int k, float scale,
                           void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
                           int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
                           void* stream) {
-    return goose_verify_step_harvest(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, draft_tok, logits, ldl, S, B,
-                                     H, Hkv, D, V, k, scale, out, lse, argmax, topk_ids, topk_vals, path, accept_len, bonus,
+    return goose_verify_step_harvest(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, n_nodes, draft_tok, logits,
+                                     ldl, S, B, H, Hkv, D, V, k, scale, out, lse, argmax, topk_ids, topk_vals, path, accept_len, bonus,
                                      new_ctx_len, nullptr, 0, nullptr, nullptr, stream);
 }
 
@@ -270,7 +271,7 @@ namespace {
 // that produce the logits next to the attention kernels (the host-buffer call uploads them on a side stream).
 int enqueue_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
                  const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
-                 const int32_t* draft_tok, const void* logits, int64_t ldl,
+                 const int32_t* n_nodes, const int32_t* draft_tok, const void* logits, int64_t ldl,
                  int S, int B, int H, int Hkv, int D, int V, int k, float scale,
                  void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
                  int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
@@ -282,12 +283,12 @@ extern "C" {
 
 int goose_verify_step_harvest(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
                               const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
-                              const int32_t* draft_tok, const void* logits, int64_t ldl,
+                              const int32_t* n_nodes, const int32_t* draft_tok, const void* logits, int64_t ldl,
                               int S, int B, int H, int Hkv, int D, int V, int k, float scale,
                               void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
                               int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
                               float* row_lse, int table_rows, int32_t* adj_ids, float* adj_scores, void* stream) {
-    return enqueue_step(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, draft_tok, logits, ldl, S, B, H, Hkv, D, V, k,
+    return enqueue_step(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, n_nodes, draft_tok, logits, ldl, S, B, H, Hkv, D, V, k,
                         scale, out, lse, argmax, topk_ids, topk_vals, path, accept_len, bonus, new_ctx_len, row_lse, table_rows,
                         adj_ids, adj_scores, stream, nullptr);
 }
@@ -297,7 +298,7 @@ int goose_verify_step_harvest(goose_ctx* c, const void* q, void* k_cache, void* 
 namespace {
 int enqueue_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int64_t kv_rows,
                  const int64_t* row_off, const int32_t* ctx_len, const int32_t* parent,
-                 const int32_t* draft_tok, const void* logits, int64_t ldl,
+                 const int32_t* n_nodes, const int32_t* draft_tok, const void* logits, int64_t ldl,
                  int S, int B, int H, int Hkv, int D, int V, int k, float scale,
                  void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
                  int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
@@ -317,8 +318,8 @@ int enqueue_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int6
     if (V < 1 || V > GOOSE_MAX_V || ldl < V || (ldl & 7) != 0 || k < 1 || k > GOOSE_MAX_K || k > V) return GOOSE_EINVAL;
     if ((long long)S * B > c->topk_rows_cap || kv_rows < 1 || kv_rows > 0x7FFFFFFFLL) return GOOSE_EINVAL;
     if (ctx_arrays_overlap(ctx_len, new_ctx_len, S)) return GOOSE_EINVAL;
-    rc = goose_tree_attn_gqa(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, S, B, H, Hkv, D, scale, out, lse,
-                             stream);
+    rc = goose_tree_attn_gqa(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, n_nodes, S, B, H, Hkv, D, scale, out,
+                             lse, stream);
     if (rc) return rc;
     // the logits are an input of the step: complete before the attention kernels above started, which do not touch
     // them -- so the top-k kernel may read them while the attention merge is still running.  With a harvest it also
@@ -328,14 +329,14 @@ int enqueue_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int6
         if (logits_ready) GOOSE_CUDA(cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), logits_ready, 0));
         cudaError_t et = goose::launch_node_topk(c, (const __nv_bfloat16*)logits, S * B, V, ldl, k, argmax, topk_ids, topk_vals,
                                                  harvest ? row_lse : nullptr, static_cast<cudaStream_t>(stream),
-                                                 /*inputs_ready=*/true);
+                                                 /*inputs_ready=*/true, n_nodes, B);
         if (et != cudaSuccess) return cuda_fail(et);
     }
     // acceptance walk + compaction in one launch (same results as goose_accept followed by goose_kv_compact); with a
     // harvest the launch also carries the table scatter: every logits row predicts the successor of its node's own draft
     // token (padding nodes carry negative tokens and are skipped)
     cudaError_t e = goose::launch_accept_compact(c, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, row_off, ctx_len,
-                                                 draft_tok, parent, argmax, S, B, Hkv, kv_rows, path, accept_len, bonus,
+                                                 draft_tok, parent, n_nodes, argmax, S, B, Hkv, kv_rows, path, accept_len, bonus,
                                                  new_ctx_len, static_cast<cudaStream_t>(stream), table_rows, k, topk_ids,
                                                  topk_vals, row_lse, harvest ? adj_ids : nullptr, adj_scores);
     if (e != cudaSuccess) return cuda_fail(e);
@@ -348,21 +349,21 @@ extern "C" {
 int goose_verify_step_host(goose_ctx* c, void* k_cache, void* v_cache, int64_t kv_rows,
                            const void* h_q, const void* h_k_new, const void* h_v_new,
                            const int64_t* h_row_off, const int32_t* h_ctx_len,
-                           const int32_t* h_parent, const int32_t* h_draft_tok, const void* h_logits,
+                           const int32_t* h_parent, const int32_t* h_n_nodes, const int32_t* h_draft_tok, const void* h_logits,
                            int S, int B, int H, int D, int V, int k, float scale,
                            void* h_out, int32_t* h_argmax, int32_t* h_topk_ids, float* h_topk_vals,
                            int32_t* h_path, int32_t* h_accept_len, int32_t* h_bonus,
                            int32_t* h_new_ctx_len, void* stream) {
     return goose_verify_step_host_gqa(c, k_cache, v_cache, kv_rows, h_q, h_k_new, h_v_new, h_row_off, h_ctx_len, h_parent,
-                                      h_draft_tok, h_logits, S, B, H, H, D, V, k, scale, h_out, h_argmax, h_topk_ids,
+                                      h_n_nodes, h_draft_tok, h_logits, S, B, H, H, D, V, k, scale, h_out, h_argmax, h_topk_ids,
                                       h_topk_vals, h_path, h_accept_len, h_bonus, h_new_ctx_len, stream);
 }
 
 int goose_verify_step_host_gqa(goose_ctx* c, void* k_cache, void* v_cache, int64_t kv_rows,
                                const void* h_q, const void* h_k_new, const void* h_v_new,
                                const int64_t* h_row_off, const int32_t* h_ctx_len,
-                               const int32_t* h_parent, const int32_t* h_draft_tok, const void* h_logits,
-                               int S, int B, int H, int Hkv, int D, int V, int k, float scale,
+                               const int32_t* h_parent, const int32_t* h_n_nodes, const int32_t* h_draft_tok,
+                               const void* h_logits, int S, int B, int H, int Hkv, int D, int V, int k, float scale,
                                void* h_out, int32_t* h_argmax, int32_t* h_topk_ids, float* h_topk_vals,
                                int32_t* h_path, int32_t* h_accept_len, int32_t* h_bonus,
                                int32_t* h_new_ctx_len, void* stream) {
@@ -377,8 +378,11 @@ int goose_verify_step_host_gqa(goose_ctx* c, void* k_cache, void* v_cache, int64
         return GOOSE_EINVAL;
     if (V < 1 || V > GOOSE_MAX_V || (V & 7) != 0 || k < 1 || k > GOOSE_MAX_K || k > V) return GOOSE_EINVAL;
     if (S == 0) return GOOSE_OK;
-    for (int s = 0; s < S; ++s)
-        if (h_row_off[s] < 0 || h_ctx_len[s] < 0 || h_row_off[s] + h_ctx_len[s] + B > kv_rows) return GOOSE_EINVAL;
+    for (int s = 0; s < S; ++s) {
+        const int nn = h_n_nodes ? h_n_nodes[s] : B;        // host data: validated here, before anything is enqueued
+        if (nn < 0 || nn > B) return GOOSE_EINVAL;
+        if (nn > 0 && (h_row_off[s] < 0 || h_ctx_len[s] < 0 || h_row_off[s] + h_ctx_len[s] + nn > kv_rows)) return GOOSE_EINVAL;
+    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
     // staging layout (256-byte aligned pieces)
@@ -392,6 +396,7 @@ int goose_verify_step_host_gqa(goose_ctx* c, void* k_cache, void* v_cache, int64
     const size_t o_ctx = off; off = up(off + S * 4);
     const size_t o_parent = off; off = up(off + rows * 4);
     const size_t o_tok = off; off = up(off + rows * 4);
+    const size_t o_nn = off; off = up(off + S * 4);
     const size_t o_argmax = off; off = up(off + rows * 4);
     const size_t o_ids = off; off = up(off + rows * k * 4);
     const size_t o_vals = off; off = up(off + rows * k * 4);
@@ -413,7 +418,7 @@ int goose_verify_step_host_gqa(goose_ctx* c, void* k_cache, void* v_cache, int64
         GOOSE_CUDA(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
         GOOSE_CUDA(cudaEventCreateWithFlags(&c->ev_logits, cudaEventDisableTiming));
     }
-    const size_t in_bytes = o_tok + rows * 4 - o_rowoff;           // row_off | ctx_len | parent | draft_tok (padded as above)
+    const size_t in_bytes = o_nn + (size_t)S * 4 - o_rowoff;       // row_off | ctx_len | parent | draft_tok | n_nodes (padded as above)
     const size_t out_bytes = o_newctx + (size_t)S * 4 - o_argmax;  // argmax | ids | vals | path | accept_len | bonus | new_ctx
     const size_t pin_need = up(in_bytes) + out_bytes;
     if (pin_need > c->pin_bytes) {
@@ -432,14 +437,17 @@ int goose_verify_step_host_gqa(goose_ctx* c, void* k_cache, void* v_cache, int64
     memcpy(pin_in + (o_ctx - o_rowoff), h_ctx_len, (size_t)S * 4);
     memcpy(pin_in + (o_parent - o_rowoff), h_parent, rows * 4);
     memcpy(pin_in + (o_tok - o_rowoff), h_draft_tok, rows * 4);
+    if (h_n_nodes) memcpy(pin_in + (o_nn - o_rowoff), h_n_nodes, (size_t)S * 4);
     GOOSE_CUDA(cudaMemcpyAsync(d + o_rowoff, pin_in, in_bytes, cudaMemcpyHostToDevice, st));
     GOOSE_CUDA(cudaMemcpyAsync(d + o_q, h_q, n_q, cudaMemcpyHostToDevice, st));
     for (int s = 0; s < S; ++s) {
+        const int nn = h_n_nodes ? h_n_nodes[s] : B;        // only the rows of nodes that exist travel
+        if (nn == 0) continue;
         size_t dst = (size_t)(h_row_off[s] + h_ctx_len[s]) * row_bytes;
         GOOSE_CUDA(cudaMemcpyAsync((char*)k_cache + dst, (const char*)h_k_new + (size_t)s * B * row_bytes,
-                                   (size_t)B * row_bytes, cudaMemcpyHostToDevice, st));
+                                   (size_t)nn * row_bytes, cudaMemcpyHostToDevice, st));
         GOOSE_CUDA(cudaMemcpyAsync((char*)v_cache + dst, (const char*)h_v_new + (size_t)s * B * row_bytes,
-                                   (size_t)B * row_bytes, cudaMemcpyHostToDevice, st));
+                                   (size_t)nn * row_bytes, cudaMemcpyHostToDevice, st));
     }
     // the logits (most of the bytes, needed by the top-k only) go up on the side stream while the attention kernels run;
     // the fork sits behind the copies above, so they have the host link to themselves and the attention starts first
@@ -448,7 +456,8 @@ int goose_verify_step_host_gqa(goose_ctx* c, void* k_cache, void* v_cache, int64
     GOOSE_CUDA(cudaMemcpyAsync(d + o_logits, h_logits, rows * V * 2, cudaMemcpyHostToDevice, c->side));
     GOOSE_CUDA(cudaEventRecord(c->ev_logits, c->side));
     rc = enqueue_step(c, d + o_q, k_cache, v_cache, kv_rows, (const int64_t*)(d + o_rowoff),
-                      (const int32_t*)(d + o_ctx), (const int32_t*)(d + o_parent), (const int32_t*)(d + o_tok),
+                      (const int32_t*)(d + o_ctx), (const int32_t*)(d + o_parent),
+                      h_n_nodes ? (const int32_t*)(d + o_nn) : nullptr, (const int32_t*)(d + o_tok),
                       d + o_logits, V, S, B, H, Hkv, D, V, k, scale, d + o_out, nullptr, (int32_t*)(d + o_argmax),
                       (int32_t*)(d + o_ids), (float*)(d + o_vals), (int32_t*)(d + o_path),
                       (int32_t*)(d + o_alen), (int32_t*)(d + o_bonus), (int32_t*)(d + o_newctx), nullptr, 0, nullptr, nullptr,

@@ -60,6 +60,17 @@ namespace goose {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Nodes of sequence s: n_nodes[s] when the array is given, else B.  The array is device data: a value outside [0, B]
+// reads as 0 (the sequence is skipped like one that has left the batch) and is reported as GOOSE_ST_BAD_NODES.
+__device__ __forceinline__ int nodes_of(const int32_t* __restrict__ n_nodes, int s, int B) {
+    if (!n_nodes) return B;
+    const int n = n_nodes[s];
+    return (n < 0 || n > B) ? 0 : n;
+}
+__device__ __forceinline__ bool nodes_bad(const int32_t* __restrict__ n_nodes, int s, int B) {
+    return n_nodes != nullptr && (n_nodes[s] < 0 || n_nodes[s] > B);
+}
+
 // Bounded mbarrier wait, shared by every kernel that waits on asynchronous copies or tensor-core commits.
 // Returns 0 when the barrier phase completed, 1 when `*abort_flag` was raised by another thread of the CTA meanwhile,
 // 2 when `limit_cycles` SM cycles passed (the caller raises the flag, records GOOSE_ST_TIMEOUT and unwinds).
@@ -95,32 +106,34 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 
 // launchers (each returns a cudaError_t from the launch)
 // inputs_ready: the logits were complete before the kernel preceding this one in the stream started (see the kernel)
+// n_nodes (may be NULL) with B: row r = s * B + i exists iff i < n_nodes[s]; other rows are neither read nor written
 cudaError_t launch_node_topk(goose_ctx* c, const __nv_bfloat16* logits, int rows, int V, int64_t ldl, int k,
                              int32_t* argmax, int32_t* ids, float* vals, float* row_lse, cudaStream_t st,
-                             bool inputs_ready = false);
+                             bool inputs_ready = false, const int32_t* n_nodes = nullptr, int B = 0);
 cudaError_t launch_harvest_scatter(goose_ctx* c, const int32_t* row_tok, int rows, int table_rows, int k,
                                    const int32_t* ids, const float* vals, const float* row_lse,
                                    int32_t* adj_ids, float* adj_scores, cudaStream_t st);
-cudaError_t launch_accept(goose_ctx* c, const int32_t* draft_tok, const int32_t* parent, const int32_t* argmax,
-                          int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus, cudaStream_t st);
+cudaError_t launch_accept(goose_ctx* c, const int32_t* draft_tok, const int32_t* parent, const int32_t* n_nodes,
+                          const int32_t* argmax, int S, int B, int32_t* path, int32_t* accept_len, int32_t* bonus,
+                          cudaStream_t st);
 cudaError_t launch_kv_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* row_off,
-                              const int32_t* ctx_len, const int32_t* path, const int32_t* accept_len,
+                              const int32_t* ctx_len, const int32_t* path, const int32_t* accept_len, const int32_t* n_nodes,
                               int S, int B, int H, int64_t kv_rows, int32_t* new_ctx, cudaStream_t st);
 cudaError_t launch_accept_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* row_off,
                                   const int32_t* ctx_len, const int32_t* draft_tok, const int32_t* parent,
-                                  const int32_t* argmax, int S, int B, int H, int64_t kv_rows, int32_t* path,
+                                  const int32_t* n_nodes, const int32_t* argmax, int S, int B, int H, int64_t kv_rows, int32_t* path,
                                   int32_t* accept_len, int32_t* bonus, int32_t* new_ctx, cudaStream_t st,
                                   int table_rows = 0, int k = 0, const int32_t* topk_ids = nullptr,
                                   const float* topk_vals = nullptr, const float* row_lse = nullptr,
                                   int32_t* adj_ids = nullptr, float* adj_scores = nullptr);
 cudaError_t launch_tree_attn_mma(goose_ctx* c, const __nv_bfloat16* q, const __nv_bfloat16* kc,
                                  const __nv_bfloat16* vc, int64_t kv_rows, const int64_t* row_off, const int32_t* ctx_len,
-                                 const int32_t* parent, int S, int B, int H, int Hkv, float scale,
+                                 const int32_t* parent, const int32_t* n_nodes, int S, int B, int H, int Hkv, float scale,
                                  __nv_bfloat16* out, float* lse, cudaStream_t st);
 cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __nv_bfloat16* kc,
                                   const __nv_bfloat16* vc, int64_t kv_rows, const int64_t* row_off,
-                                  const int32_t* ctx_len, const int32_t* parent, int S, int B, int H, int Hkv,
-                                  float scale, __nv_bfloat16* out, float* lse, cudaStream_t st);
+                                  const int32_t* ctx_len, const int32_t* parent, const int32_t* n_nodes, int S, int B, int H,
+                                  int Hkv, float scale, __nv_bfloat16* out, float* lse, cudaStream_t st);
 
 cudaError_t launch_bounded_wait_selftest(goose_ctx* c, long long limit_cycles, int32_t* result, cudaStream_t st);
 

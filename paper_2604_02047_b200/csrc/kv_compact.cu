@@ -17,6 +17,7 @@ __global__ void __launch_bounds__(kCompactThreads)
 kv_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc,
                   const int64_t* __restrict__ row_off, const int32_t* __restrict__ ctx_len,
                   const int32_t* __restrict__ path, const int32_t* __restrict__ accept_len,
+                  const int32_t* __restrict__ n_nodes,
                   int B, int row_vec /* 16-byte vectors per row = H*128*2/16 */, int64_t kv_rows,
                   int32_t* __restrict__ new_ctx, int32_t* __restrict__ status) {
     __shared__ int s_path[kMaxB];
@@ -27,19 +28,27 @@ kv_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc,
     pdl_wait();
     pdl_trigger();
     const int ctx = ctx_len[s];
+    const int nn = nodes_of(n_nodes, s, B);              // nodes of this sequence's tree; 0: it has left the batch
+    if (nn == 0) {                                       // nothing moves, nothing is appended
+        if (blockIdx.x == 0 && which == 0 && threadIdx.x == 0) {
+            new_ctx[s] = ctx;
+            if (nodes_bad(n_nodes, s, B)) atomicOr(&status[s], GOOSE_ST_BAD_NODES);
+        }
+        return;
+    }
     int L = accept_len[s];
     if (threadIdx.x == 0) s_bad = 0;
     __syncthreads();
     // rows this sequence owns must lie inside the cache: never form an address from unchecked device data
     const int64_t r0 = row_off[s];
-    const bool bad_rows = ctx < 0 || r0 < 0 || r0 + ctx + B > kv_rows;
-    bool bad = (L < 0 || L >= B) || bad_rows;
+    const bool bad_rows = ctx < 0 || r0 < 0 || r0 + ctx + nn > kv_rows;
+    bool bad = (L < 0 || L >= nn) || bad_rows;
     if (!bad) {
         for (int j = threadIdx.x; j <= L; j += kCompactThreads) {
             int pj = path[(size_t)s * B + j];
             s_path[j] = pj;
             int prev = (j == 0) ? -1 : path[(size_t)s * B + j - 1];
-            if (pj < j || pj >= B || pj <= prev || (j == 0 && pj != 0)) s_bad = 1;
+            if (pj < j || pj >= nn || pj <= prev || (j == 0 && pj != 0)) s_bad = 1;
         }
     }
     __syncthreads();
@@ -68,13 +77,13 @@ kv_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc,
 }
 
 cudaError_t launch_kv_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* row_off,
-                              const int32_t* ctx_len, const int32_t* path, const int32_t* accept_len,
+                              const int32_t* ctx_len, const int32_t* path, const int32_t* accept_len, const int32_t* n_nodes,
                               int S, int B, int H, int64_t kv_rows, int32_t* new_ctx, cudaStream_t st) {
     if (S == 0) return cudaSuccess;
     int row_vec = H * kHeadDim * 2 / 16;
     dim3 grid((row_vec + kCompactThreads - 1) / kCompactThreads, 2, S);
     cudaError_t e = launch_pdl(kv_compact_kernel, grid, dim3(kCompactThreads), 0, st, kc, vc, row_off, ctx_len, path,
-                               accept_len, B, row_vec, kv_rows, new_ctx, c->status);
+                               accept_len, n_nodes, B, row_vec, kv_rows, new_ctx, c->status);
     c->launches++;
     return e;
 }
@@ -91,7 +100,8 @@ cudaError_t launch_kv_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc
 __global__ void __launch_bounds__(kCompactThreads)
 accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __restrict__ row_off,
                       const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ draft_tok,
-                      const int32_t* __restrict__ parent, const int32_t* __restrict__ argmax,
+                      const int32_t* __restrict__ parent, const int32_t* __restrict__ n_nodes,
+                      const int32_t* __restrict__ argmax,
                       int B, int row_vec, int64_t kv_rows, int32_t* __restrict__ path,
                       int32_t* __restrict__ accept_len, int32_t* __restrict__ bonus, int32_t* __restrict__ new_ctx,
                       int32_t* __restrict__ status,
@@ -101,6 +111,9 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
     __shared__ int s_path[kMaxB];
     __shared__ int s_len;
     const int s = blockIdx.z;
+    // n_nodes[] is an input of the step like parent[] and the tokens: read ahead of the wait.  nn = nodes of this
+    // sequence's tree; 0: the sequence has left the batch and nothing of it is read or moved.
+    const int nn = nodes_of(n_nodes, s, B);
     if (blockIdx.y == 2) {
         // ---- harvest scatter role
         const int lane = threadIdx.x & 31;
@@ -108,11 +121,14 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
         const size_t r = (size_t)s * B + i;
         int tok = -1;
         bool write = false;
-        if (i < B) {
+        if (i < nn) {
             tok = draft_tok[r];
             if (tok >= 0 && tok < table_rows) {
-                bool later = false;                        // does a later row carry the same token?
-                for (int j = (int)r + 1 + lane; j < rows_total; j += 32) later |= (draft_tok[j] == tok);
+                bool later = false;                        // does a later row (of a node that exists) carry the same token?
+                for (int j = (int)r + 1 + lane; j < rows_total; j += 32) {
+                    const int sj = j / B;
+                    if (j - sj * B < nodes_of(n_nodes, sj, B)) later |= (draft_tok[j] == tok);
+                }
                 write = !__any_sync(0xFFFFFFFFu, later);
             }
         }
@@ -135,7 +151,7 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
     // rows this sequence owns must lie inside the cache: never form an address from unchecked device data
     const int ctx0 = ctx_len[s];
     const int64_t r0 = row_off[s];
-    const bool bad_rows = ctx0 < 0 || r0 < 0 || r0 + ctx0 + B > kv_rows;
+    const bool bad_rows = nn > 0 && (ctx0 < 0 || r0 < 0 || r0 + ctx0 + nn > kv_rows);
     constexpr int kPer = kMaxB / 32;
     int my_par[kPer], my_tok[kPer];
     bool bad = false;
@@ -148,7 +164,7 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
             const int c = lane + 32 * t;
             my_par[t] = -2;
             my_tok[t] = -1;
-            if (c < B) {
+            if (c < nn) {
                 const int pp = par[c];
                 my_par[t] = pp;
                 my_tok[t] = tok[c];
@@ -156,7 +172,7 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
             }
         }
         bad = __any_sync(0xFFFFFFFFu, bad);
-        for (int c = lane; c < B; c += 32) s_path[c] = (c == 0) ? 0 : -1;
+        for (int c = lane; c < B; c += 32) s_path[c] = (c == 0 && nn > 0) ? 0 : -1;
     }
     pdl_wait();
     pdl_trigger();
@@ -168,13 +184,13 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
         for (int t = 0; t < kPer; ++t) my_match[t] = false;
         __syncwarp();
         int v = 0, len = 0;
-        if (!bad) {
+        if (!bad && nn > 0) {
 #pragma unroll
             for (int t = 0; t < kPer; ++t) {
                 const int c = lane + 32 * t;
-                if (c >= 1 && c < B) my_match[t] = (my_tok[t] == am[my_par[t]]);
+                if (c >= 1 && c < nn) my_match[t] = (my_tok[t] == am[my_par[t]]);
             }
-            for (int step = 0; step < B - 1; ++step) {
+            for (int step = 0; step < nn - 1; ++step) {
                 int cand = 0x7FFFFFFF;
 #pragma unroll
                 for (int t = kPer - 1; t >= 0; --t)
@@ -192,10 +208,11 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
             for (int c = lane; c < B; c += 32) path[(size_t)s * B + c] = s_path[c];
             if (lane == 0) {
                 accept_len[s] = len;
-                bonus[s] = bad ? -1 : am[v];
-                new_ctx[s] = ctx0 + 1 + len;
+                bonus[s] = (bad || nn == 0) ? -1 : am[v];
+                new_ctx[s] = nn == 0 ? ctx0 : ctx0 + 1 + len;
                 if (bad) atomicOr(&status[s], GOOSE_ST_BAD_PARENT);
                 if (bad_rows) atomicOr(&status[s], GOOSE_ST_BAD_ROWS);
+                if (nodes_bad(n_nodes, s, B)) atomicOr(&status[s], GOOSE_ST_BAD_NODES);
             }
         }
     }
@@ -220,7 +237,7 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
 
 cudaError_t launch_accept_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* row_off,
                                   const int32_t* ctx_len, const int32_t* draft_tok, const int32_t* parent,
-                                  const int32_t* argmax, int S, int B, int H, int64_t kv_rows, int32_t* path,
+                                  const int32_t* n_nodes, const int32_t* argmax, int S, int B, int H, int64_t kv_rows, int32_t* path,
                                   int32_t* accept_len, int32_t* bonus, int32_t* new_ctx, cudaStream_t st,
                                   int table_rows, int k, const int32_t* topk_ids, const float* topk_vals,
                                   const float* row_lse, int32_t* adj_ids, float* adj_scores) {
@@ -234,7 +251,7 @@ cudaError_t launch_accept_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16
     }
     dim3 grid(gx, scatter ? 3 : 2, S);
     cudaError_t e = launch_pdl(accept_compact_kernel, grid, dim3(kCompactThreads), 0, st, kc, vc, row_off, ctx_len,
-                               draft_tok, parent, argmax, B, row_vec, kv_rows, path, accept_len, bonus, new_ctx, c->status,
+                               draft_tok, parent, n_nodes, argmax, B, row_vec, kv_rows, path, accept_len, bonus, new_ctx, c->status,
                                S * B, table_rows, k, topk_ids, topk_vals, row_lse, adj_ids, adj_scores);
     c->launches++;
     return e;

@@ -70,11 +70,11 @@ __device__ __forceinline__ uint32_t topk_smem_u32(const void* p) { return (uint3
 // pass sums exp(x - chunk max) over every element, chunks are merged like split softmax partials.
 template <int KCAP, bool LSE>
 __global__ void __launch_bounds__(kTopkThreads, 1)
-node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items, int V, int64_t ldl, int k, int chunks,
+node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items_all, int V, int64_t ldl, int k, int chunks,
                  u64* __restrict__ ws_cand, int32_t* __restrict__ row_counters,
                  int32_t* __restrict__ argmax, int32_t* __restrict__ ids, float* __restrict__ vals,
                  float* __restrict__ row_lse, float2* __restrict__ ws_lse, int32_t* __restrict__ status,
-                 int inputs_ready) {
+                 int inputs_ready, const int32_t* __restrict__ n_nodes, int S, int B) {
     extern __shared__ __align__(128) unsigned char s_stage[];   // kTopkStages x 64 KB
     __shared__ u64 s_full[kTopkStages];
     __shared__ float s_sum[32];
@@ -93,8 +93,6 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items, int 
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int G = gridDim.x;
-    const long long w_begin = items * blockIdx.x / G, w_end = items * (blockIdx.x + 1) / G;
-    const int n_local = (int)(w_end - w_begin);
     if (tid == 0) {
         for (int i = 0; i < kTopkStages; ++i)
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(topk_smem_u32(&s_full[i])));
@@ -110,6 +108,27 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items, int 
     bool waited = inputs_ready == 0;
     if (waited) pdl_wait();
     pdl_trigger();
+    // Per-sequence node counts (n_nodes != NULL; rows = S * B, row s * B + i belongs to node i of sequence s): rows of
+    // nodes that do not exist are left out of the item list, so their logits are never read.  The list then runs over
+    // the rows that exist, numbered densely ("row" below; the cross-CTA scratch is indexed by it), and row_of() gives
+    // the row in memory.  n_nodes[] is an input like the logits: it may be read ahead of the dependency wait.
+    long long items = items_all;
+    if (n_nodes) {
+        long long live = 0;
+        for (int s = 0; s < S; ++s) live += nodes_of(n_nodes, s, B);
+        items = live * chunks;
+    }
+    auto row_of = [&](long long r) -> long long {
+        if (!n_nodes) return r;
+        for (int s = 0; s < S; ++s) {
+            const int n = nodes_of(n_nodes, s, B);
+            if (r < n) return (long long)s * B + r;
+            r -= n;
+        }
+        return 0;                                        // not reached: r is below the number of live rows
+    };
+    const long long w_begin = items * blockIdx.x / G, w_end = items * (blockIdx.x + 1) / G;
+    const int n_local = (int)(w_end - w_begin);
 
     const unsigned short* lg = reinterpret_cast<const unsigned short*>(logits);
     // thread 0: stream item j of this CTA into stage j % kTopkStages (the copy is rounded up to 16 bytes, which
@@ -124,7 +143,7 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items, int 
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(topk_smem_u32(bar)), "r"(bytes) : "memory");
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                      ::"r"(topk_smem_u32(s_stage + (j % kTopkStages) * kTopkStageBytes)),
-                       "l"(lg + (size_t)row * ldl + base), "r"(bytes), "r"(topk_smem_u32(bar)) : "memory");
+                       "l"(lg + (size_t)row_of(row) * ldl + base), "r"(bytes), "r"(topk_smem_u32(bar)) : "memory");
     };
     int issued = 0;
     if (tid == 0)
@@ -189,13 +208,14 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items, int 
             for (int o = 16; o > 0; o >>= 1) csum += __shfl_xor_sync(0xFFFFFFFFu, csum, o);
         }
         if (chunks == 1) {                               // the chunk is the row: write it out
+            const size_t out_row = (size_t)row_of(pend_row);
             if (lane < k) {
                 const int32_t id = (int32_t)(0xFFFFu - (mine & 0xFFFFu));
-                ids[(size_t)pend_row * k + lane] = id;
-                if (vals) vals[(size_t)pend_row * k + lane] = value_of_sortable16(mine >> 16);
-                if (lane == 0) argmax[pend_row] = id;
+                ids[out_row * k + lane] = id;
+                if (vals) vals[out_row * k + lane] = value_of_sortable16(mine >> 16);
+                if (lane == 0) argmax[out_row] = id;
             }
-            if (LSE && lane == 0) row_lse[pend_row] = cmax + logf(csum);
+            if (LSE && lane == 0) row_lse[out_row] = cmax + logf(csum);
             return;
         }
         const bool part_begins = (pend_j == 0) || (pend_chunk == 0);
@@ -299,13 +319,14 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items, int 
                 fin_m = M; fin_s = sum;
             }
         }
+        const size_t out_row = (size_t)row_of(pend_row);
         if (lane < k) {
             const int32_t id = (int32_t)(0xFFFFFFFFu - (uint32_t)(win & 0xFFFFFFFFull));
-            ids[(size_t)pend_row * k + lane] = id;
-            if (vals) vals[(size_t)pend_row * k + lane] = value_of_sortable16((uint32_t)(win >> 32));
-            if (lane == 0) argmax[pend_row] = id;
+            ids[out_row * k + lane] = id;
+            if (vals) vals[out_row * k + lane] = value_of_sortable16((uint32_t)(win >> 32));
+            if (lane == 0) argmax[out_row] = id;
         }
-        if (LSE && lane == 0) row_lse[pend_row] = fin_m + logf(fin_s);
+        if (LSE && lane == 0) row_lse[out_row] = fin_m + logf(fin_s);
     };
 
     for (int j = 0; j < n_local; ++j) {
@@ -479,21 +500,23 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items, int 
         if (++chunk == chunks) { chunk = 0; ++row; }
     }
     if (warp == 0 && pend_chunk >= 0) finish_pending();  // the CTA's last item
-    if (!waited) pdl_wait();                             // (every CTA has at least one item, so warp 0 has waited)
+    if (!waited) pdl_wait();                             // a CTA without items, or the warps that wrote nothing
 }
 
 namespace {
 template <int KCAP, bool LSE>
 cudaError_t launch_topk_inst(int grid, cudaStream_t st, const __nv_bfloat16* logits, long long items, int V, int64_t ldl,
                              int k, int chunks, u64* ws, int32_t* counters, int32_t* argmax, int32_t* ids, float* vals,
-                             float* row_lse, float2* ws_lse, int32_t* status, int inputs_ready) {
+                             float* row_lse, float2* ws_lse, int32_t* status, int inputs_ready, const int32_t* n_nodes, int S,
+                             int B) {
     return launch_pdl(node_topk_kernel<KCAP, LSE>, dim3(grid), dim3(kTopkThreads), kTopkSmem, st, logits, items, V, ldl, k,
-                      chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status, inputs_ready);
+                      chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status, inputs_ready, n_nodes, S, B);
 }
 
 cudaError_t launch_topk_any(int num_sms, cudaStream_t st, const __nv_bfloat16* logits, int rows, int V, int64_t ldl, int k,
                             u64* ws, int32_t* counters, int32_t* argmax, int32_t* ids, float* vals, float* row_lse,
-                            float2* ws_lse, int32_t* status, int inputs_ready) {
+                            float2* ws_lse, int32_t* status, int inputs_ready, const int32_t* n_nodes = nullptr, int B = 0) {
+    const int S = (n_nodes && B > 0) ? rows / B : 0;
     const int chunks = (V + kTopkChunk - 1) / kTopkChunk;
     const long long items = (long long)rows * chunks;
     // every CTA gets q = ceil(items / SMs) items or one fewer; using the fewest CTAs that q allows loses no time and
@@ -501,10 +524,10 @@ cudaError_t launch_topk_any(int num_sms, cudaStream_t st, const __nv_bfloat16* l
     const long long q = (items + num_sms - 1) / num_sms;
     const int grid = (int)((items + q - 1) / q);
     if (row_lse)
-        return k <= 8 ? launch_topk_inst<8, true>(grid, st, logits, items, V, ldl, k, chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status, inputs_ready)
-                      : launch_topk_inst<16, true>(grid, st, logits, items, V, ldl, k, chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status, inputs_ready);
-    return k <= 8 ? launch_topk_inst<8, false>(grid, st, logits, items, V, ldl, k, chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status, inputs_ready)
-                  : launch_topk_inst<16, false>(grid, st, logits, items, V, ldl, k, chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status, inputs_ready);
+        return k <= 8 ? launch_topk_inst<8, true>(grid, st, logits, items, V, ldl, k, chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status, inputs_ready, n_nodes, S, B)
+                      : launch_topk_inst<16, true>(grid, st, logits, items, V, ldl, k, chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status, inputs_ready, n_nodes, S, B);
+    return k <= 8 ? launch_topk_inst<8, false>(grid, st, logits, items, V, ldl, k, chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status, inputs_ready, n_nodes, S, B)
+                  : launch_topk_inst<16, false>(grid, st, logits, items, V, ldl, k, chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status, inputs_ready, n_nodes, S, B);
 }
 }  // namespace
 
@@ -520,10 +543,11 @@ cudaError_t init_topk_kernel() {
 
 cudaError_t launch_node_topk(goose_ctx* c, const __nv_bfloat16* logits, int rows, int V, int64_t ldl, int k,
                              int32_t* argmax, int32_t* ids, float* vals, float* row_lse, cudaStream_t st,
-                             bool inputs_ready) {
+                             bool inputs_ready, const int32_t* n_nodes, int B) {
     if (rows == 0) return cudaSuccess;
     cudaError_t e = launch_topk_any(c->num_sms, st, logits, rows, V, ldl, k, c->topk_cand, c->row_counters, argmax, ids, vals,
-                                    row_lse, reinterpret_cast<float2*>(c->topk_lse_ws), c->status, inputs_ready ? 1 : 0);
+                                    row_lse, reinterpret_cast<float2*>(c->topk_lse_ws), c->status, inputs_ready ? 1 : 0,
+                                    n_nodes, B);
     c->launches++;
     return e;
 }

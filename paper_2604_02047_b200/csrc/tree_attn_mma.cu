@@ -87,7 +87,7 @@ __global__ void __launch_bounds__(256)
 tree_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ kc,
                      const __nv_bfloat16* __restrict__ vc, const int64_t* __restrict__ row_off,
                      const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ parent,
-                     int B, int H, int Hkv, int64_t kv_rows, float scale_log2, int splits,
+                     const int32_t* __restrict__ n_nodes, int Bcap, int H, int Hkv, int64_t kv_rows, float scale_log2, int splits,
                      float* __restrict__ partials, int32_t* __restrict__ head_counters,
                      int32_t* __restrict__ status, __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -101,13 +101,20 @@ tree_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     const int hk = h / (H / Hkv);
     pdl_wait();
     pdl_trigger();
+    // B = nodes of THIS sequence's tree (n_nodes[s] <= Bcap, the stride of q / out / parent); nodes beyond it do not
+    // exist: nothing of theirs is read, their output rows are not written, their cache rows are past the last key
+    const int B = nodes_of(n_nodes, s, Bcap);
+    if (B == 0) {                                          // the sequence has left the batch (every CTA of it agrees)
+        if (tid == 0 && split == 0 && h == 0 && nodes_bad(n_nodes, s, Bcap)) atomicOr(&status[s], GOOSE_ST_BAD_NODES);
+        return;
+    }
     const int ctx = max(ctx_len[s], 0);                    // device data: a negative length is treated as 0
     const int64_t row0 = row_off[s];
     const int n_keys = ctx + B;
     const int n_tiles = (n_keys + kKT - 1) / kKT;
     const int t_begin = (int)((long long)n_tiles * split / splits);
     const int t_end = (int)((long long)n_tiles * (split + 1) / splits);
-    const int32_t* par = parent + (size_t)s * B;
+    const int32_t* par = parent + (size_t)s * Bcap;
 
     // ---- validate parent[] (every CTA of the sequence reaches the same verdict)
     int bad = 0;
@@ -129,8 +136,8 @@ tree_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
     for (int n = 0; n < 16; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
 
     if (warp_active) {
-        const uint32_t* qA = reinterpret_cast<const uint32_t*>(q + (((size_t)s * B + (rowA < B ? rowA : 0)) * H + h) * kHeadDim);
-        const uint32_t* qB = reinterpret_cast<const uint32_t*>(q + (((size_t)s * B + (rowB < B ? rowB : 0)) * H + h) * kHeadDim);
+        const uint32_t* qA = reinterpret_cast<const uint32_t*>(q + (((size_t)s * Bcap + (rowA < B ? rowA : 0)) * H + h) * kHeadDim);
+        const uint32_t* qB = reinterpret_cast<const uint32_t*>(q + (((size_t)s * Bcap + (rowB < B ? rowB : 0)) * H + h) * kHeadDim);
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
             qf[ks][0] = rowA < B ? qA[ks * 8 + t4] : 0u;
@@ -240,8 +247,8 @@ tree_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
             // zero-fill this CTA's share of the head's output
             for (int idx = tid + split * nthreads; idx < B * (kHeadDim / 2); idx += nthreads * splits) {
                 int i = idx / (kHeadDim / 2), c = idx % (kHeadDim / 2);
-                reinterpret_cast<uint32_t*>(out + (((size_t)s * B + i) * H + h) * kHeadDim)[c] = 0u;
-                if (lse && c == 0) lse[((size_t)s * B + i) * H + h] = 0.f;
+                reinterpret_cast<uint32_t*>(out + (((size_t)s * Bcap + i) * H + h) * kHeadDim)[c] = 0u;
+                if (lse && c == 0) lse[((size_t)s * Bcap + i) * H + h] = 0.f;
             }
             return;
         }
@@ -250,13 +257,13 @@ tree_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
 #pragma unroll
             for (int n = 0; n < 16; ++n) {
                 if (rowA < B)
-                    *reinterpret_cast<uint32_t*>(out + (((size_t)s * B + rowA) * H + h) * kHeadDim + 8 * n + 2 * t4) = pack_bf16(o[n][0] * iA, o[n][1] * iA);
+                    *reinterpret_cast<uint32_t*>(out + (((size_t)s * Bcap + rowA) * H + h) * kHeadDim + 8 * n + 2 * t4) = pack_bf16(o[n][0] * iA, o[n][1] * iA);
                 if (rowB < B)
-                    *reinterpret_cast<uint32_t*>(out + (((size_t)s * B + rowB) * H + h) * kHeadDim + 8 * n + 2 * t4) = pack_bf16(o[n][2] * iB, o[n][3] * iB);
+                    *reinterpret_cast<uint32_t*>(out + (((size_t)s * Bcap + rowB) * H + h) * kHeadDim + 8 * n + 2 * t4) = pack_bf16(o[n][2] * iB, o[n][3] * iB);
             }
             if (lse && t4 == 0) {
-                if (rowA < B) lse[((size_t)s * B + rowA) * H + h] = (mA + log2f(lA)) * kLn2;
-                if (rowB < B) lse[((size_t)s * B + rowB) * H + h] = (mB + log2f(lB)) * kLn2;
+                if (rowA < B) lse[((size_t)s * Bcap + rowA) * H + h] = (mA + log2f(lA)) * kLn2;
+                if (rowB < B) lse[((size_t)s * Bcap + rowB) * H + h] = (mB + log2f(lB)) * kLn2;
             }
         }
         return;
@@ -301,8 +308,8 @@ tree_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* _
             a0 += w * ov.x; a1 += w * ov.y;
         }
         float inv = 1.f / L;
-        reinterpret_cast<uint32_t*>(out + (((size_t)s * B + i) * H + h) * kHeadDim)[c] = pack_bf16(a0 * inv, a1 * inv);
-        if (lse && c == 0) lse[((size_t)s * B + i) * H + h] = (M + log2f(L)) * kLn2;
+        reinterpret_cast<uint32_t*>(out + (((size_t)s * Bcap + i) * H + h) * kHeadDim)[c] = pack_bf16(a0 * inv, a1 * inv);
+        if (lse && c == 0) lse[((size_t)s * Bcap + i) * H + h] = (M + log2f(L)) * kLn2;
     }
 }
 
@@ -322,7 +329,7 @@ int mma_splits(const goose_ctx* c, int S, int H) {
 
 cudaError_t launch_tree_attn_mma(goose_ctx* c, const __nv_bfloat16* q, const __nv_bfloat16* kc,
                                  const __nv_bfloat16* vc, int64_t kv_rows, const int64_t* row_off, const int32_t* ctx_len,
-                                 const int32_t* parent, int S, int B, int H, int Hkv, float scale,
+                                 const int32_t* parent, const int32_t* n_nodes, int S, int B, int H, int Hkv, float scale,
                                  __nv_bfloat16* out, float* lse, cudaStream_t st) {
     if (S == 0 || H == 0) return cudaSuccess;
     int splits = mma_splits(c, S, H);
@@ -330,7 +337,7 @@ cudaError_t launch_tree_attn_mma(goose_ctx* c, const __nv_bfloat16* q, const __n
     if (warps < 4) warps = 4;
     dim3 grid(splits, H, S);
     cudaError_t e = launch_pdl(tree_attn_mma_kernel, grid, dim3(warps * 32), kMmaSmem, st, q, kc, vc, row_off, ctx_len,
-                               parent, B, H, Hkv, kv_rows, scale * kLog2e, splits, c->partials, c->head_counters, c->status, out, lse);
+                               parent, n_nodes, B, H, Hkv, kv_rows, scale * kLog2e, splits, c->partials, c->head_counters, c->status, out, lse);
     c->launches++;
     return e;
 }

@@ -208,11 +208,16 @@ __device__ __forceinline__ bool group_sync(Header* hd, uint32_t& n, int32_t* sta
 // ---------------------------------------------------------------- work partition (same code in every role)
 struct Work {
     const int32_t* ctx_len;
+    const int32_t* n_nodes;   // per-sequence node counts, or NULL (every tree has B nodes)
     int S, H, B, G;           // H = heads of the work list = M tiles x key/value heads (M-tile-major)
     long long total;          // all items
     bool small;               // total * (G + 1) fits 31 bits: 32-bit arithmetic (64-bit division is slow on the GPU)
-    // ctx_len comes from device memory: a negative value is treated as 0 (the tree rows alone)
-    __device__ __forceinline__ int tiles(int s) const { return (max(ctx_len[s], 0) + B + kTile - 1) / kTile; }
+    // ctx_len comes from device memory: a negative value is treated as 0 (the tree rows alone).  A sequence's keys are
+    // its prefix and the nodes its tree really has; a sequence without nodes (it has left the batch) has no items.
+    __device__ __forceinline__ int tiles(int s) const {
+        const int nn = nodes_of(n_nodes, s, B);
+        return nn == 0 ? 0 : (max(ctx_len[s], 0) + nn + kTile - 1) / kTile;
+    }
     __device__ __forceinline__ void init() {
         long long tot = 0;
         for (int s = 0; s < S; ++s) tot += (long long)H * tiles(s);
@@ -253,7 +258,10 @@ struct Cursor {               // walks items in order
         ++w; ++t;
         if (t == T) {
             t = 0; ++h;
-            if (h == wk.H) { h = 0; ++s; if (s < wk.S) T = wk.tiles(s); }
+            if (h == wk.H) {                              // next sequence that has any items
+                h = 0; ++s;
+                while (s < wk.S && (T = wk.tiles(s)) == 0) ++s;
+            }
         }
     }
 };
@@ -266,6 +274,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                       const __grid_constant__ CUtensorMap tmap_v, const int64_t* __restrict__ row_off,
                       const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ parent,
+                      const int32_t* __restrict__ n_nodes,
                       int S, int B, int H, int Hkv_arg, int g_arg, int nb_arg, int64_t kv_rows, float scale_log2,
                       float* __restrict__ partials,
                       int32_t* __restrict__ status,
@@ -310,10 +319,13 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     // one (the combine kernel) get resident early -- it waits for this grid before reading the partials
     pdl_wait();
     pdl_trigger();
+    if (n_nodes && blockIdx.x == 0 && threadIdx.x == 33)   // an idle lane reports node counts outside [0, B] (read as 0)
+        for (int s = 0; s < S; ++s)
+            if (nodes_bad(n_nodes, s, B)) atomicOr(&status[s], GOOSE_ST_BAD_NODES);
     Work wk;
     // g query heads per key/value head, nb nodes per M tile (nb * g <= 128), n_mt M tiles per sequence
     const int n_mt = kGrouped ? (B + nb - 1) / nb : 1;
-    wk.ctx_len = ctx_len; wk.S = S; wk.H = n_mt * Hkv; wk.B = B; wk.G = gridDim.x;
+    wk.ctx_len = ctx_len; wk.n_nodes = n_nodes; wk.S = S; wk.H = n_mt * Hkv; wk.B = B; wk.G = gridDim.x;
     wk.init();
     const long long w_begin = wk.cta_start(blockIdx.x), w_end = wk.cta_start(blockIdx.x + 1);
 
@@ -446,10 +458,11 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 const int s0 = cu.s, h0 = cu.h, T = cu.T;
                 const int mt = kGrouped ? h0 / Hkv : 0, hk = h0 - mt * Hkv;
                 const int node = mt * nb + i_local;        // tree node of this thread's row
-                const bool row_valid = i_local < nb && node < B;
-                const bool warp_has_rows = 32 * (warp & 3) < min(nb, B - mt * nb) * g;
+                const int nn = nodes_of(n_nodes, s0, B);   // nodes this sequence's tree really has (> 0: it has items)
+                const bool row_valid = i_local < nb && node < nn;
+                const bool warp_has_rows = 32 * (warp & 3) < min(nb, nn - mt * nb) * g;
                 const int ctx = max(ctx_len[s0], 0);
-                const int n_keys = ctx + B;
+                const int n_keys = ctx + nn;               // rows behind may hold anything: masked, and zeroed in V
                 const int32_t* par = parent + (size_t)s0 * B;
                 const int t_first = cu.t;
                 // new sequence: validate parent[] (all 128 threads reach the same verdict) and rebuild
@@ -457,7 +470,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                 const bool new_seq = s0 != cur_s;
                 if (new_seq) {
                     cur_s = s0;
-                    if (row < B) {                         // thread r stages parent[r] (independent of the row stacking)
+                    if (row < nn) {                        // thread r stages parent[r] (independent of the row stacking)
                         int p = par[row];
                         hd->par[row] = p;
                         if ((row == 0) ? (p != -1) : (p < 0 || p >= row)) hd->bad_parent = 1;
@@ -465,7 +478,7 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                     // the sequence's rows must lie inside the cache (TMA would only read zeros outside, but the
                     // result would be meaningless): treated like an invalid tree, with its own status bit
                     const int64_t r0 = row_off[s0];
-                    const bool bad_rows = ctx_len[s0] < 0 || r0 < 0 || r0 + ctx + B > kv_rows;
+                    const bool bad_rows = ctx_len[s0] < 0 || r0 < 0 || r0 + ctx + nn > kv_rows;
                     if (bad_rows && sm_tid == 0) { hd->bad_parent = 1; atomicOr(&status[s0], GOOSE_ST_BAD_ROWS); }
                     ok = group_sync(hd, gsync, status);
                     bad = hd->bad_parent != 0;
@@ -689,7 +702,8 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
 // Lane <-> row (coalesced float4 loads of the transposed partial layout), warp <-> 16 output columns.
 template <bool kGrouped>
 __global__ void __launch_bounds__(kCombineThreads)
-tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, int S, int B, int H, int Hkv_arg, int g_arg, int nb_arg, int G,
+tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ n_nodes, int S, int B, int H,
+                         int Hkv_arg, int g_arg, int nb_arg, int G,
                          const float* __restrict__ partials, __nv_bfloat16* __restrict__ out,
                          float* __restrict__ lse) {
     const int Hkv = kGrouped ? Hkv_arg : H, g = kGrouped ? g_arg : 1, nb = kGrouped ? nb_arg : B;
@@ -700,19 +714,19 @@ tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, int S, int B, int 
     // kernel triggers its dependents after its own pdl_wait(), i.e. after whatever produced ctx_len[] completed.
     // So all of it runs before the wait, and the partial loads are issued the moment the main grid is done.
     Work wk;
-    wk.ctx_len = ctx_len; wk.S = S; wk.H = Hw; wk.B = B; wk.G = G;
+    wk.ctx_len = ctx_len; wk.n_nodes = n_nodes; wk.S = S; wk.H = Hw; wk.B = B; wk.G = G;
     wk.init();
     long long off = 0;
     for (int ss = 0; ss < s; ++ss) off += (long long)Hw * wk.tiles(ss);
-    const int T = wk.tiles(s);
+    const int T = wk.tiles(s);                             // 0: the sequence has no nodes, hence no items and no output
     const long long head_first = off + (long long)h * T;
-    const int c_lo = wk.cta_of(head_first), c_hi = wk.cta_of(head_first + T - 1);
-    const bool whole = c_lo == c_hi;                       // written directly by the main kernel
+    const int c_lo = T > 0 ? wk.cta_of(head_first) : 0, c_hi = T > 0 ? wk.cta_of(head_first + T - 1) : 0;
+    const bool whole = c_lo == c_hi;                       // written directly by the main kernel (or nothing to write)
     const int row = rg * 32 + lane;                        // row of the M tile = (node of the tile, head of the group)
     const int mt = kGrouped ? h / Hkv : 0, hk = h - mt * Hkv;
     const int i_local = kGrouped ? row / g : row, node = mt * nb + i_local;
     const int hq = hk * g + (row - i_local * g);
-    const bool row_valid = i_local < nb && node < B;
+    const bool row_valid = i_local < nb && node < nodes_of(n_nodes, s, B);
     // CTA c's partial for this head sits in slot 2c, or 2c+1 when its segment starts at the head's first tile,
     // which only the first CTA can do.  With fewer items than CTAs some CTAs in [c_lo, c_hi] are empty.
     const int flag_lo = wk.cta_start(c_lo) <= head_first ? 1 : 0;
@@ -863,8 +877,8 @@ int auto_attn_impl(const goose_ctx* c, int S, int B, int H) {
 
 cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __nv_bfloat16* kc,
                                   const __nv_bfloat16* vc, int64_t kv_rows, const int64_t* row_off,
-                                  const int32_t* ctx_len, const int32_t* parent, int S, int B, int H, int Hkv,
-                                  float scale, __nv_bfloat16* out, float* lse, cudaStream_t st) {
+                                  const int32_t* ctx_len, const int32_t* parent, const int32_t* n_nodes, int S, int B, int H,
+                                  int Hkv, float scale, __nv_bfloat16* out, float* lse, cudaStream_t st) {
     if (!c->encode_tiled) return cudaErrorNotSupported;
     if (S == 0) return cudaSuccess;
     const int g = H / Hkv;                              // query heads per key/value head (validated by the caller)
@@ -879,14 +893,14 @@ cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __
     if (2 * grid > c->n_slots) grid = c->n_slots / 2;
     const bool grouped = g > 1;
     cudaError_t e = launch_pdl(grouped ? tree_attn_umma_kernel<true> : tree_attn_umma_kernel<false>, dim3(grid),
-                               dim3(kThreads), kUmmaSmem, st, mq, mk, mv, row_off, ctx_len, parent, S, B, H, Hkv, g, nb,
+                               dim3(kThreads), kUmmaSmem, st, mq, mk, mv, row_off, ctx_len, parent, n_nodes, S, B, H, Hkv, g, nb,
                                kv_rows, scale * kLog2e, c->partials, c->status, out, lse);
     c->launches++;
     if (e != cudaSuccess) return e;
     dim3 cgrid((nb * g + 31) / 32, n_mt * Hkv, S);
     const float* parts = c->partials;
     e = launch_pdl(grouped ? tree_attn_combine_kernel<true> : tree_attn_combine_kernel<false>, cgrid,
-                   dim3(kCombineThreads), 0, st, ctx_len, S, B, H, Hkv, g, nb, grid, parts, out, lse);
+                   dim3(kCombineThreads), 0, st, ctx_len, n_nodes, S, B, H, Hkv, g, nb, grid, parts, out, lse);
     c->launches++;
     return e;
 }

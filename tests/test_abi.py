@@ -36,7 +36,7 @@ def test_strerror_and_null_context(lib):
     # argument errors are caught on the host before any CUDA call
     assert lib.goose_set_attn_impl(None, 0) == -1
     assert lib.goose_destroy(None) == -1
-    assert lib.goose_node_topk(None, None, 0, 0, ctypes.c_int64(0), 0, None, None, None, None) == -1
+    assert lib.goose_node_topk(None, None, 0, 0, ctypes.c_int64(0), 0, None, 0, None, None, None, None) == -1
     out = ctypes.c_void_p()
     assert lib.goose_create(ctypes.byref(out), 0, 0, 128, 32, 128) == -1      # max_S < 1
     assert lib.goose_create(ctypes.byref(out), 0, 1, 129, 32, 128) == -1      # max_B > 128

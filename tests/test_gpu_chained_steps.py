@@ -123,6 +123,6 @@ def test_new_ctx_len_must_not_alias_ctx_len(goose):
     path = torch.zeros((1, 8), dtype=torch.int32, device="cuda"); alen = torch.zeros(1, dtype=torch.int32, device="cuda")
     rc = lib.goose_kv_compact(goose.h, binding._p(d["k_cache"]), binding._p(d["v_cache"]), ctypes.c_int64(48),
                               binding._p(d["row_off"]), binding._p(d["ctx_len"]), binding._p(path), binding._p(alen),
-                              ctypes.c_int(1), ctypes.c_int(8), ctypes.c_int(2), ctypes.c_int(128),
+                              binding._p(None), ctypes.c_int(1), ctypes.c_int(8), ctypes.c_int(2), ctypes.c_int(128),
                               binding._p(d["ctx_len"]), binding._stream())
     assert rc == -1

@@ -129,7 +129,7 @@ def test_step_with_harvest_argument_errors():
     def call(row_lse, adj_ids, adj_sc, vals, table_rows):
         return g.lib.goose_verify_step_harvest(
             g.h, P(d["q"]), P(d["k_cache"]), P(d["v_cache"]), ctypes.c_int64(d["k_cache"].shape[0]), P(d["row_off"]),
-            P(d["ctx_len"]), P(d["parent"]), P(d["draft_tok"]), P(d["logits"]), ctypes.c_int64(x.V), ctypes.c_int(x.S),
+            P(d["ctx_len"]), P(d["parent"]), P(None), P(d["draft_tok"]), P(d["logits"]), ctypes.c_int64(x.V), ctypes.c_int(x.S),
             ctypes.c_int(x.B), ctypes.c_int(x.H), ctypes.c_int(x.H), ctypes.c_int(128), ctypes.c_int(x.V), ctypes.c_int(x.k),
             ctypes.c_float(x.scale), P(o["out"]), None, P(o["argmax"]), P(o["topk_ids"]), P(vals), P(o["path"]),
             P(o["accept_len"]), P(o["bonus"]), P(o["new_ctx_len"]), P(row_lse), ctypes.c_int(table_rows), P(adj_ids), P(adj_sc),

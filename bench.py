@@ -37,6 +37,8 @@ METRIC = "tree_verify_steps_per_s"
 UNIT = "steps/s"
 L2_BYTES = 126 * 1024 * 1024
 MIN_REGIONS = 5                 # the K-step timed region is repeated at least this often
+BURST_GAP_S = 0.2               # idle time in front of every burst region (the part cools back to its full clocks)
+BURST_MS = 10.0                 # length of a burst region of the per-kernel legs
 SUSTAIN_SECONDS = 1.5           # further regions keep the GPU under the same load until the clock sampler has >= 10 samples
 # DRAM traffic per attention call (main + merge kernels) from the ncu captures summarised under profiles/ (bytes); these
 # are NOT measured by the run that prints them: `roofline.traffic_source` names the capture.  None = not captured.
@@ -68,9 +70,10 @@ class ClockSampler:
                   "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
     NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
-    def __init__(self, gpu_index: int, uuid: str = None, period_s: float = 0.02):
+    def __init__(self, gpu_index: int, uuid: str = None, period_s: float = 0.004):
         self.gpu, self.uuid, self.period = gpu_index, uuid, period_s
         self.samples = []               # (sm_mhz, max_mhz, [reason flags])
+        self.active = True              # samples are recorded only while this is set (the idle gaps between bursts are not)
         self._stop = threading.Event()
         self._t = None
         self._nvml = None
@@ -109,10 +112,11 @@ class ClockSampler:
 
     def _run(self):
         while not self._stop.is_set():
-            try:
-                self._sample_nvml() if self._nvml else self._sample_smi()
-            except Exception:
-                pass
+            if self.active:
+                try:
+                    self._sample_nvml() if self._nvml else self._sample_smi()
+                except Exception:
+                    pass
             self._stop.wait(self.period if self._nvml else 0.1)
 
     def __enter__(self):
@@ -310,6 +314,7 @@ def quick_step_timing(config_id, dev, peak, uuid):
             step(i)
         stream.synchronize()
         with ClockSampler(dev.index, uuid) as clk:
+            clk.active = False
             for name, fn in (("step", step), ("attn", attn), ("topk", topk)):
                 gr = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(gr, stream=stream, capture_error_mode="thread_local"):
@@ -318,8 +323,14 @@ def quick_step_timing(config_id, dev, peak, uuid):
                 for _ in range(2):
                     gr.replay()
                 one = _time_graph(gr, 1, stream)
-                rounds = int(max(1, min(400, 0.05e3 / max(one, 1e-3))))      # about 50 ms per region
-                regs = [_time_graph(gr, rounds, stream) / (rounds * R) for _ in range(MIN_REGIONS)]
+                rounds = int(max(1, min(400, BURST_MS / max(one, 1e-3))))    # bursts of about BURST_MS behind an idle gap
+                regs = []
+                for _ in range(MIN_REGIONS):
+                    clk.active = False
+                    time.sleep(BURST_GAP_S)
+                    clk.active = True
+                    regs.append(_time_graph(gr, rounds, stream) / (rounds * R))
+                    clk.active = False
                 res[name] = (float(np.median(regs)), float(min(regs)))
     ab = synth.algorithmic_bytes(x.S, x.H, x.B, x.D, x.V, x.ctx_len, Hkv=x.Hkv)
     g.close()
@@ -449,25 +460,37 @@ def run_ours(args, x, cfg, rank, world, local_rank):
 
         for _ in range(max(1, -(-args.warmup // R))):     # warm-up replays
             g_step.replay()
-        def leg(gr, rounds):
-            _time_graph(gr, 1, stream)
-            regs = [_time_graph(gr, rounds, stream) / (rounds * R) for _ in range(MIN_REGIONS)]
+        def burst(clk, fn):
+            """One burst region: an idle gap, then the timed work with the clock sampler recording."""
+            clk.active = False
+            time.sleep(BURST_GAP_S)
+            clk.active = True
+            ms = fn()
+            clk.active = False
+            return ms
+
+        def leg(clk, gr, gap=True):
+            one = max(_time_graph(gr, 1, stream), 1e-3)
+            rounds = int(max(1, min(400, BURST_MS / one)))
+            regs = [(burst(clk, lambda: _time_graph(gr, rounds, stream)) if gap else _time_graph(gr, rounds, stream)) / (rounds * R)
+                    for _ in range(MIN_REGIONS)]
             return float(np.median(regs)), float(min(regs))
 
-        # Phase 1 (burst, the way the HBM peak itself was measured): the MIN_REGIONS official regions, then each kernel
-        # alone.  Phase 2 (sustained): the same step replayed for SUSTAIN_SECONDS more, where a 1 kW part may meet its
-        # power cap, then the attention call once more under that load.  The clock sampler runs through both.
+        # Phase 1 (bursts, the way the HBM copy peak itself was measured -- the best of ten 0.6 ms copies): MIN_REGIONS
+        # regions of K steps, each behind an idle gap, then each kernel alone in bursts of about BURST_MS.  Phase 2
+        # (sustained): the same step replayed back to back for --sustain-seconds, where a 1 kW part meets its power cap,
+        # then the attention call once more under that load.  The clock sampler records inside the regions only.
         with ClockSampler(local_rank, uuid) as clk_burst:
-            region_ms = [region() for _ in range(MIN_REGIONS)]
+            clk_burst.active = False
+            region_ms = [burst(clk_burst, region) for _ in range(MIN_REGIONS)]
             local_ms = float(np.median(region_ms))
-            leg_rounds = max(1, min(200, int(0.03e3 / max(local_ms / args.steps, 1e-3)) // R + 1))    # about 30 ms a region
-            legs = {name: leg(gr, leg_rounds) for name, gr in (("attn", g_attn), ("topk", g_topk), ("harv", g_harv), ("sh", g_sh))}
+            legs = {name: leg(clk_burst, gr) for name, gr in (("attn", g_attn), ("topk", g_topk), ("harv", g_harv), ("sh", g_sh))}
         with ClockSampler(local_rank, uuid) as clk_sus:
-            t_end = time.perf_counter() + SUSTAIN_SECONDS
+            t_end = time.perf_counter() + args.sustain_seconds
             sustain_ms = []
             while time.perf_counter() < t_end and len(sustain_ms) < 20000:
                 sustain_ms.append(region())
-            legs["attn_sustained"] = leg(g_attn, leg_rounds)
+            legs["attn_sustained"] = leg(clk_sus, g_attn, gap=False)
         clocks_burst, clocks_sus = clk_burst.summary(), clk_sus.summary()
         both = ClockSampler.__new__(ClockSampler)
         both.samples, both._nvml = clk_burst.samples + clk_sus.samples, clk_burst._nvml
@@ -528,10 +551,11 @@ def run_ours(args, x, cfg, rank, world, local_rank):
         "config": workload_config(x, cfg.name),
         "protocol": {"l2": "rotating %d input replicas (%.2f GB total, > 2x L2)" % (R, R * footprint / 1e9),
                      "timing": "CUDA graph replay of whole steps, CUDA events around each region of K steps, barrier + "
-                               "synchronize on both sides, max over ranks; ms_per_step = median region",
+                               "synchronize on both sides, max over ranks; ms_per_step = median region; every region "
+                               "starts behind %.1f s of idle time (burst, as the copy peak was taken)" % BURST_GAP_S,
                      "regions": MIN_REGIONS, "ms_per_step_min": min_ms,
                      "sustained_regions": len(sustain_ms), "sustained_ms_per_step": sustain_ms_step,
-                     "sustained_note": "the same K-step region repeated for %.1f s after the headline regions" % SUSTAIN_SECONDS,
+                     "sustained_note": "the same K-step region repeated for %.1f s after the headline regions" % args.sustain_seconds,
                      "multi_gpu": "replicas only"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                 "steps": e2e_steps, "regions": MIN_REGIONS, "us_per_step": e2e_ms * 1e3 / e2e_steps,
@@ -548,9 +572,9 @@ def run_ours(args, x, cfg, rank, world, local_rank):
                      "algorithmic_bytes": ab["attn"], "us_per_launch": attn_ms * 1e3, "us_per_launch_min": legs["attn"][1] * 1e3,
                      "us_per_launch_sustained": legs["attn_sustained"][0] * 1e3,
                      "frac_sustained": ab["attn"] / (legs["attn_sustained"][0] * 1e-3) / 1e9 / peak,
-                     "note": "frac: the attention call timed alone in bursts of about 30 ms right after the headline regions, as "
-                             "the copy peak was (clocks.burst); frac_sustained: the same after SUSTAIN_SECONDS of "
-                             "continuous load (clocks.sustained, where sw_power_cap may be active)"},
+                     "note": "frac: the attention call timed alone, median of %d bursts of about %d ms each behind %.1f s of idle "
+                             "time, as the copy peak was taken (clocks.burst); frac_sustained: the same back to back after "
+                             "the sustained phase (clocks.sustained, where sw_power_cap is active)" % (MIN_REGIONS, BURST_MS, BURST_GAP_S)},
         "kernels": {"tree_attn_us": attn_ms * 1e3, "node_topk_us": topk_ms * 1e3, "harvest_us": harv_ms * 1e3,
                     "step_with_harvest_us": sh_ms * 1e3,
                     "node_topk_gbs": ab["topk"] / (topk_ms * 1e-3) / 1e9,
@@ -605,6 +629,8 @@ def main():
     ap.add_argument("--dry-run", action="store_true", help="rank plumbing only, stub step, no GPU (CPU tests of the N > 1 path)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--sustain-seconds", type=float, default=SUSTAIN_SECONDS,
+                    help="length of the sustained phase behind the headline regions (0 for profiling runs)")
     ap.add_argument("--no-others", action="store_true",
                     help="skip the short timings of the other four workloads that the default line carries as context")
     args = ap.parse_args()

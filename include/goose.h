@@ -164,8 +164,8 @@ int goose_harvest(goose_ctx* ctx, const void* logits, int rows, int V, int64_t l
  *     rows <= GOOSE_STATIC_TOPK_MAX_ROWS, otherwise GOOSE_EINVAL (nothing is enqueued).
  *   - It calls no cudaMalloc / cudaFree and no allocating library routine.  The first call on each
  *     device looks up the device address of the array (cudaGetSymbolAddress, with that device current),
- *     reads the device's multiprocessor count and sets the kernel's shared-memory attribute; make that
- *     first call outside any stream capture.
+ *     reads the device's multiprocessor count and sets the kernel's shared-memory attribute (host-side
+ *     queries, made once per device).
  *   - All calls share the one array, which keeps the contents of the previous call; the counters it
  *     needs at zero are cleared on `stream` before the kernel.  Two calls whose kernels may overlap on
  *     the GPU (different streams, no dependency between them) race on the array: serialise them.

@@ -441,6 +441,7 @@ def run_ours(args, x, cfg, rank, world, local_rank):
         g_topk, _ = capture(topk)
         g_harv, _ = capture(harvest)
         g_sh, _ = capture(step_harvest)
+        g_warm, _ = capture(lambda i: step(0), 8)         # one replica over and over (8 steps per replay): the L2-warm figure
 
         def region():
             """EXACTLY K steps between two events, barrier + synchronize on both sides; returns this rank's ms."""
@@ -485,6 +486,7 @@ def run_ours(args, x, cfg, rank, world, local_rank):
             region_ms = [burst(clk_burst, region) for _ in range(MIN_REGIONS)]
             local_ms = float(np.median(region_ms))
             legs = {name: leg(clk_burst, gr) for name, gr in (("attn", g_attn), ("topk", g_topk), ("harv", g_harv), ("sh", g_sh))}
+            legs["warm"] = tuple(v * R / 8 for v in leg(clk_burst, g_warm))  # leg() divides by R steps per replay; here it is 8
         with ClockSampler(local_rank, uuid) as clk_sus:
             t_end = time.perf_counter() + args.sustain_seconds
             sustain_ms = []
@@ -577,6 +579,9 @@ def run_ours(args, x, cfg, rank, world, local_rank):
                              "the sustained phase (clocks.sustained, where sw_power_cap is active)" % (MIN_REGIONS, BURST_MS, BURST_GAP_S)},
         "kernels": {"tree_attn_us": attn_ms * 1e3, "node_topk_us": topk_ms * 1e3, "harvest_us": harv_ms * 1e3,
                     "step_with_harvest_us": sh_ms * 1e3,
+                    "step_l2_warm_us": legs["warm"][0] * 1e3,
+                    "step_l2_warm_note": "the same input replica every replay, so whatever of its footprint fits stays in L2; "
+                                         "context only, the metric is the L2-cold rotation",
                     "node_topk_gbs": ab["topk"] / (topk_ms * 1e-3) / 1e9,
                     "step_gbs": ab["total"] / (ms_per_step * 1e-3) / 1e9,
                     "step_frac_of_peak": ab["total"] / (ms_per_step * 1e-3) / 1e9 / peak},

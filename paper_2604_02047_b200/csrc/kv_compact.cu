@@ -13,6 +13,8 @@ namespace goose {
 constexpr int kCompactThreads = 128;
 constexpr int kCompactBatch = 8;
 
+// kCounts = false is the instantiation for n_nodes == NULL
+template <bool kCounts>
 __global__ void __launch_bounds__(kCompactThreads)
 kv_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc,
                   const int64_t* __restrict__ row_off, const int32_t* __restrict__ ctx_len,
@@ -20,6 +22,8 @@ kv_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc,
                   const int32_t* __restrict__ n_nodes,
                   int B, int row_vec /* 16-byte vectors per row = H*128*2/16 */, int64_t kv_rows,
                   int32_t* __restrict__ new_ctx, int32_t* __restrict__ status) {
+    if (!kCounts) n_nodes = nullptr;
+
     __shared__ int s_path[kMaxB];
     __shared__ int s_bad;
     const int s = blockIdx.z;
@@ -82,7 +86,7 @@ cudaError_t launch_kv_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc
     if (S == 0) return cudaSuccess;
     int row_vec = H * kHeadDim * 2 / 16;
     dim3 grid((row_vec + kCompactThreads - 1) / kCompactThreads, 2, S);
-    cudaError_t e = launch_pdl(kv_compact_kernel, grid, dim3(kCompactThreads), 0, st, kc, vc, row_off, ctx_len, path,
+    cudaError_t e = launch_pdl(n_nodes ? kv_compact_kernel<true> : kv_compact_kernel<false>, grid, dim3(kCompactThreads), 0, st, kc, vc, row_off, ctx_len, path,
                                accept_len, n_nodes, B, row_vec, kv_rows, new_ctx, c->status);
     c->launches++;
     return e;
@@ -97,6 +101,7 @@ cudaError_t launch_kv_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc
 // With a harvest (adj_ids != NULL) the launch carries a third block role, blockIdx.y == 2: one warp per logits row of the
 // sequence writes that row's top-k ids and softmax scores to adjacency-table row draft_tok[row] unless a later row of the
 // call carries the same token -- the rule of harvest_scatter_kernel, decided here before the wait (tokens are inputs).
+template <bool kCounts>
 __global__ void __launch_bounds__(kCompactThreads)
 accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __restrict__ row_off,
                       const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ draft_tok,
@@ -108,12 +113,15 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
                       int rows_total, int table_rows, int k, const int32_t* __restrict__ topk_ids,
                       const float* __restrict__ topk_vals, const float* __restrict__ row_lse,
                       int32_t* __restrict__ adj_ids, float* __restrict__ adj_scores) {
+    if (!kCounts) n_nodes = nullptr;
+
     __shared__ int s_path[kMaxB];
     __shared__ int s_len;
     const int s = blockIdx.z;
     // n_nodes[] is an input of the step like parent[] and the tokens: read ahead of the wait.  nn = nodes of this
     // sequence's tree; 0: the sequence has left the batch and nothing of it is read or moved.
-    const int nn = nodes_of(n_nodes, s, B);
+    const int nn = kCounts ? nodes_of(n_nodes, s, B) : B;
+    const bool live = !kCounts || nn > 0;               // (without counts every sequence has its B nodes)
     if (blockIdx.y == 2) {
         // ---- harvest scatter role
         const int lane = threadIdx.x & 31;
@@ -126,6 +134,7 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
             if (tok >= 0 && tok < table_rows) {
                 bool later = false;                        // does a later row (of a node that exists) carry the same token?
                 for (int j = (int)r + 1 + lane; j < rows_total; j += 32) {
+                    if (!kCounts) { later |= (draft_tok[j] == tok); continue; }
                     const int sj = j / B;
                     if (j - sj * B < nodes_of(n_nodes, sj, B)) later |= (draft_tok[j] == tok);
                 }
@@ -151,7 +160,7 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
     // rows this sequence owns must lie inside the cache: never form an address from unchecked device data
     const int ctx0 = ctx_len[s];
     const int64_t r0 = row_off[s];
-    const bool bad_rows = nn > 0 && (ctx0 < 0 || r0 < 0 || r0 + ctx0 + nn > kv_rows);
+    const bool bad_rows = live && (ctx0 < 0 || r0 < 0 || r0 + ctx0 + nn > kv_rows);
     constexpr int kPer = kMaxB / 32;
     int my_par[kPer], my_tok[kPer];
     bool bad = false;
@@ -172,7 +181,7 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
             }
         }
         bad = __any_sync(0xFFFFFFFFu, bad);
-        for (int c = lane; c < B; c += 32) s_path[c] = (c == 0 && nn > 0) ? 0 : -1;
+        for (int c = lane; c < B; c += 32) s_path[c] = (c == 0 && live) ? 0 : -1;
     }
     pdl_wait();
     pdl_trigger();
@@ -184,7 +193,7 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
         for (int t = 0; t < kPer; ++t) my_match[t] = false;
         __syncwarp();
         int v = 0, len = 0;
-        if (!bad && nn > 0) {
+        if (!bad && live) {
 #pragma unroll
             for (int t = 0; t < kPer; ++t) {
                 const int c = lane + 32 * t;
@@ -208,11 +217,11 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
             for (int c = lane; c < B; c += 32) path[(size_t)s * B + c] = s_path[c];
             if (lane == 0) {
                 accept_len[s] = len;
-                bonus[s] = (bad || nn == 0) ? -1 : am[v];
-                new_ctx[s] = nn == 0 ? ctx0 : ctx0 + 1 + len;
+                bonus[s] = (bad || !live) ? -1 : am[v];
+                new_ctx[s] = !live ? ctx0 : ctx0 + 1 + len;
                 if (bad) atomicOr(&status[s], GOOSE_ST_BAD_PARENT);
                 if (bad_rows) atomicOr(&status[s], GOOSE_ST_BAD_ROWS);
-                if (nodes_bad(n_nodes, s, B)) atomicOr(&status[s], GOOSE_ST_BAD_NODES);
+                if (kCounts && nodes_bad(n_nodes, s, B)) atomicOr(&status[s], GOOSE_ST_BAD_NODES);
             }
         }
     }
@@ -250,7 +259,7 @@ cudaError_t launch_accept_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16
         if (sx > gx) gx = sx;
     }
     dim3 grid(gx, scatter ? 3 : 2, S);
-    cudaError_t e = launch_pdl(accept_compact_kernel, grid, dim3(kCompactThreads), 0, st, kc, vc, row_off, ctx_len,
+    cudaError_t e = launch_pdl(n_nodes ? accept_compact_kernel<true> : accept_compact_kernel<false>, grid, dim3(kCompactThreads), 0, st, kc, vc, row_off, ctx_len,
                                draft_tok, parent, n_nodes, argmax, B, row_vec, kv_rows, path, accept_len, bonus, new_ctx, c->status,
                                S * B, table_rows, k, topk_ids, topk_vals, row_lse, adj_ids, adj_scores);
     c->launches++;

@@ -68,7 +68,8 @@ __device__ __forceinline__ uint32_t topk_smem_u32(const void* p) { return (uint3
 
 // LSE = true additionally returns the row's log-sum-exp (for the softmax scores of the harvest): the second
 // pass sums exp(x - chunk max) over every element, chunks are merged like split softmax partials.
-template <int KCAP, bool LSE>
+// COUNTS = false is the instantiation for n_nodes == NULL (the item list is known before the dependency wait)
+template <int KCAP, bool LSE, bool COUNTS>
 __global__ void __launch_bounds__(kTopkThreads, 1)
 node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items_all, int V, int64_t ldl, int k, int chunks,
                  u64* __restrict__ ws_cand, int32_t* __restrict__ row_counters,
@@ -93,6 +94,9 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items_all, 
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int G = gridDim.x;
+    if (!COUNTS) n_nodes = nullptr;
+    long long items = items_all;
+    long long w_begin = items * blockIdx.x / G, w_end = items * (blockIdx.x + 1) / G;   // final when !COUNTS
     if (tid == 0) {
         for (int i = 0; i < kTopkStages; ++i)
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(topk_smem_u32(&s_full[i])));
@@ -112,14 +116,14 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items_all, 
     // nodes that do not exist are left out of the item list, so their logits are never read.  The list then runs over
     // the rows that exist, numbered densely ("row" below; the cross-CTA scratch is indexed by it), and row_of() gives
     // the row in memory.  n_nodes[] is an input like the logits: it may be read ahead of the dependency wait.
-    long long items = items_all;
-    if (n_nodes) {
+    if (COUNTS && n_nodes) {
         long long live = 0;
         for (int s = 0; s < S; ++s) live += nodes_of(n_nodes, s, B);
         items = live * chunks;
+        w_begin = items * blockIdx.x / G; w_end = items * (blockIdx.x + 1) / G;
     }
     auto row_of = [&](long long r) -> long long {
-        if (!n_nodes) return r;
+        if (!COUNTS || !n_nodes) return r;
         for (int s = 0; s < S; ++s) {
             const int n = nodes_of(n_nodes, s, B);
             if (r < n) return (long long)s * B + r;
@@ -127,7 +131,6 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items_all, 
         }
         return 0;                                        // not reached: r is below the number of live rows
     };
-    const long long w_begin = items * blockIdx.x / G, w_end = items * (blockIdx.x + 1) / G;
     const int n_local = (int)(w_end - w_begin);
 
     const unsigned short* lg = reinterpret_cast<const unsigned short*>(logits);
@@ -509,7 +512,8 @@ cudaError_t launch_topk_inst(int grid, cudaStream_t st, const __nv_bfloat16* log
                              int k, int chunks, u64* ws, int32_t* counters, int32_t* argmax, int32_t* ids, float* vals,
                              float* row_lse, float2* ws_lse, int32_t* status, int inputs_ready, const int32_t* n_nodes, int S,
                              int B) {
-    return launch_pdl(node_topk_kernel<KCAP, LSE>, dim3(grid), dim3(kTopkThreads), kTopkSmem, st, logits, items, V, ldl, k,
+    return launch_pdl(n_nodes ? node_topk_kernel<KCAP, LSE, true> : node_topk_kernel<KCAP, LSE, false>, dim3(grid),
+                      dim3(kTopkThreads), kTopkSmem, st, logits, items, V, ldl, k,
                       chunks, ws, counters, argmax, ids, vals, row_lse, ws_lse, status, inputs_ready, n_nodes, S, B);
 }
 
@@ -534,10 +538,14 @@ cudaError_t launch_topk_any(int num_sms, cudaStream_t st, const __nv_bfloat16* l
 
 // per-device kernel attributes: the stage ring needs the opt-in shared-memory size
 cudaError_t init_topk_kernel() {
-    cudaError_t e = cudaFuncSetAttribute(node_topk_kernel<8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTopkSmem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(node_topk_kernel<16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTopkSmem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(node_topk_kernel<8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTopkSmem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(node_topk_kernel<16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTopkSmem);
+    cudaError_t e = cudaSuccess;
+    auto opt_in = [&](const void* fn) {
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kTopkSmem);
+    };
+    opt_in((const void*)node_topk_kernel<8, false, false>);  opt_in((const void*)node_topk_kernel<8, false, true>);
+    opt_in((const void*)node_topk_kernel<16, false, false>); opt_in((const void*)node_topk_kernel<16, false, true>);
+    opt_in((const void*)node_topk_kernel<8, true, false>);   opt_in((const void*)node_topk_kernel<8, true, true>);
+    opt_in((const void*)node_topk_kernel<16, true, false>);  opt_in((const void*)node_topk_kernel<16, true, true>);
     return e;
 }
 

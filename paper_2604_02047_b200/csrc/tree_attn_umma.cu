@@ -215,6 +215,7 @@ struct Work {
     // ctx_len comes from device memory: a negative value is treated as 0 (the tree rows alone).  A sequence's keys are
     // its prefix and the nodes its tree really has; a sequence without nodes (it has left the batch) has no items.
     __device__ __forceinline__ int tiles(int s) const {
+        if (!n_nodes) return (max(ctx_len[s], 0) + B + kTile - 1) / kTile;
         const int nn = nodes_of(n_nodes, s, B);
         return nn == 0 ? 0 : (max(ctx_len[s], 0) + nn + kTile - 1) / kTile;
     }
@@ -260,7 +261,8 @@ struct Cursor {               // walks items in order
             t = 0; ++h;
             if (h == wk.H) {                              // next sequence that has any items
                 h = 0; ++s;
-                while (s < wk.S && (T = wk.tiles(s)) == 0) ++s;
+                if (!wk.n_nodes) { if (s < wk.S) T = wk.tiles(s); }
+                else while (s < wk.S && (T = wk.tiles(s)) == 0) ++s;
             }
         }
     }
@@ -269,7 +271,8 @@ struct Cursor {               // walks items in order
 // ---------------------------------------------------------------- the kernel
 // kGrouped = false is multi-head attention: one query head per key/value head and one M tile per sequence are
 // compile-time facts there (the per-row index arithmetic folds away); kGrouped = true takes them from the arguments.
-template <bool kGrouped>
+// kCounts = false is the instantiation for n_nodes == NULL: the counts fold away at compile time
+template <bool kGrouped, bool kCounts>
 __global__ void __launch_bounds__(kThreads, 1)
 tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                       const __grid_constant__ CUtensorMap tmap_v, const int64_t* __restrict__ row_off,
@@ -279,6 +282,8 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
                       float* __restrict__ partials,
                       int32_t* __restrict__ status,
                       __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+    if (!kCounts) n_nodes = nullptr;
+
     const int Hkv = kGrouped ? Hkv_arg : H, g = kGrouped ? g_arg : 1, nb = kGrouped ? nb_arg : B;
     extern __shared__ unsigned char smem_raw[];
     Header* hd = reinterpret_cast<Header*>(smem_raw);
@@ -700,12 +705,14 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
 // main kernel covered entirely was written directly and is skipped; any other is the merge of its CTAs' partials:
 //   M = max m_p,  L = sum l_p 2^(m_p - M),  out = sum_p 2^(m_p - M) O_p / L.
 // Lane <-> row (coalesced float4 loads of the transposed partial layout), warp <-> 16 output columns.
-template <bool kGrouped>
+template <bool kGrouped, bool kCounts>
 __global__ void __launch_bounds__(kCombineThreads)
 tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ n_nodes, int S, int B, int H,
                          int Hkv_arg, int g_arg, int nb_arg, int G,
                          const float* __restrict__ partials, __nv_bfloat16* __restrict__ out,
                          float* __restrict__ lse) {
+    if (!kCounts) n_nodes = nullptr;
+
     const int Hkv = kGrouped ? Hkv_arg : H, g = kGrouped ? g_arg : 1, nb = kGrouped ? nb_arg : B;
     const int rg = blockIdx.x, h = blockIdx.y, s = blockIdx.z;   // h = head of the work list (M tile, KV head)
     const int Hw = gridDim.y;
@@ -720,7 +727,8 @@ tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, const int32_t* __r
     for (int ss = 0; ss < s; ++ss) off += (long long)Hw * wk.tiles(ss);
     const int T = wk.tiles(s);                             // 0: the sequence has no nodes, hence no items and no output
     const long long head_first = off + (long long)h * T;
-    const int c_lo = T > 0 ? wk.cta_of(head_first) : 0, c_hi = T > 0 ? wk.cta_of(head_first + T - 1) : 0;
+    const bool any = !kCounts || T > 0;                    // (without counts every sequence has tiles)
+    const int c_lo = any ? wk.cta_of(head_first) : 0, c_hi = any ? wk.cta_of(head_first + T - 1) : 0;
     const bool whole = c_lo == c_hi;                       // written directly by the main kernel (or nothing to write)
     const int row = rg * 32 + lane;                        // row of the M tile = (node of the tile, head of the group)
     const int mt = kGrouped ? h / Hkv : 0, hk = h - mt * Hkv;
@@ -862,9 +870,13 @@ cudaError_t launch_bounded_wait_selftest(goose_ctx* c, long long limit_cycles, i
 }
 
 cudaError_t init_umma_kernel() {
-    cudaError_t e = cudaFuncSetAttribute(tree_attn_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmem);
+    cudaError_t e = cudaFuncSetAttribute(tree_attn_umma_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmem);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(tree_attn_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmem);
+    e = cudaFuncSetAttribute(tree_attn_umma_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(tree_attn_umma_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(tree_attn_umma_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmem);
 }
 
 int auto_attn_impl(const goose_ctx* c, int S, int B, int H) {
@@ -892,14 +904,19 @@ cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __
     int grid = c->num_sms;
     if (2 * grid > c->n_slots) grid = c->n_slots / 2;
     const bool grouped = g > 1;
-    cudaError_t e = launch_pdl(grouped ? tree_attn_umma_kernel<true> : tree_attn_umma_kernel<false>, dim3(grid),
+    const bool counts = n_nodes != nullptr;
+    auto main_kernel = grouped ? (counts ? tree_attn_umma_kernel<true, true> : tree_attn_umma_kernel<true, false>)
+                               : (counts ? tree_attn_umma_kernel<false, true> : tree_attn_umma_kernel<false, false>);
+    auto merge_kernel = grouped ? (counts ? tree_attn_combine_kernel<true, true> : tree_attn_combine_kernel<true, false>)
+                                : (counts ? tree_attn_combine_kernel<false, true> : tree_attn_combine_kernel<false, false>);
+    cudaError_t e = launch_pdl(main_kernel, dim3(grid),
                                dim3(kThreads), kUmmaSmem, st, mq, mk, mv, row_off, ctx_len, parent, n_nodes, S, B, H, Hkv, g, nb,
                                kv_rows, scale * kLog2e, c->partials, c->status, out, lse);
     c->launches++;
     if (e != cudaSuccess) return e;
     dim3 cgrid((nb * g + 31) / 32, n_mt * Hkv, S);
     const float* parts = c->partials;
-    e = launch_pdl(grouped ? tree_attn_combine_kernel<true> : tree_attn_combine_kernel<false>, cgrid,
+    e = launch_pdl(merge_kernel, cgrid,
                    dim3(kCombineThreads), 0, st, ctx_len, n_nodes, S, B, H, Hkv, g, nb, grid, parts, out, lse);
     c->launches++;
     return e;

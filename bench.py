@@ -42,8 +42,8 @@ BURST_MS = 10.0                 # length of a burst region of the per-kernel leg
 SUSTAIN_SECONDS = 1.5           # further regions keep the GPU under the same load until the clock sampler has >= 10 samples
 # DRAM traffic per attention call (main + merge kernels) from the ncu captures summarised under profiles/ (bytes); these
 # are NOT measured by the run that prints them: `roofline.traffic_source` names the capture.  None = not captured.
-NCU_TRAFFIC_BYTES = {"33b": (227_500_000, "profiles/tree_attn_umma_33b.md"),      # 223.31 MB read + 4.05-4.31 MB written
-                     "13b": (89_330_000, "profiles/tree_attn_umma_13b.md"),       # 86.43 MB read + 2.80-3.00 MB written
+NCU_TRAFFIC_BYTES = {"33b": (227_200_000, "profiles/tree_attn_umma_33b.md"),      # 223.29 MB read + 3.89-3.95 MB written
+                     "13b": (89_230_000, "profiles/tree_attn_umma_13b.md"),       # 86.42 MB read + 2.65-2.98 MB written
                      "gqa8b": (169_570_000, "profiles/tree_attn_umma_gqa8b.md")}  # 165.0 MB read + 3.2-5.8 MB written
 
 

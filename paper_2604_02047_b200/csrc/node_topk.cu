@@ -123,13 +123,17 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items_all, 
         w_begin = items * blockIdx.x / G; w_end = items * (blockIdx.x + 1) / G;
     }
     auto row_of = [&](long long r) -> long long {
-        if (!COUNTS || !n_nodes) return r;
-        for (int s = 0; s < S; ++s) {
-            const int n = nodes_of(n_nodes, s, B);
-            if (r < n) return (long long)s * B + r;
-            r -= n;
+        if constexpr (!COUNTS) {
+            return r;
+        } else {
+            if (!n_nodes) return r;
+            for (int s = 0; s < S; ++s) {
+                const int n = nodes_of(n_nodes, s, B);
+                if (r < n) return (long long)s * B + r;
+                r -= n;
+            }
+            return 0;                                    // not reached: r is below the number of live rows
         }
-        return 0;                                        // not reached: r is below the number of live rows
     };
     const int n_local = (int)(w_end - w_begin);
 

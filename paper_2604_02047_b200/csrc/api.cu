@@ -4,6 +4,7 @@
 #include <new>
 
 #include "goose_internal.cuh"
+#include "tree_attn_combine.cuh"
 
 namespace {
 
@@ -318,9 +319,27 @@ int enqueue_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int6
     if (V < 1 || V > GOOSE_MAX_V || ldl < V || (ldl & 7) != 0 || k < 1 || k > GOOSE_MAX_K || k > V) return GOOSE_EINVAL;
     if ((long long)S * B > c->topk_rows_cap || kv_rows < 1 || kv_rows > 0x7FFFFFFFLL) return GOOSE_EINVAL;
     if (ctx_arrays_overlap(ctx_len, new_ctx_len, S)) return GOOSE_EINVAL;
-    rc = goose_tree_attn_gqa(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, n_nodes, S, B, H, Hkv, D, scale, out,
-                             lse, stream);
-    if (rc) return rc;
+    // Attention.  With the tensor-core kernel the merge of its split heads does not get a launch of its own here: it
+    // rides in the step's last launch, beside the walk and the compaction, so the top-k starts the moment the main
+    // kernel's CTAs leave their SMs (out[] and lse[] are complete when the step is).
+    goose::CombinePlan merge_plan;
+    merge_plan.valid = false;
+    if (!(scale > 0.f) || !(scale < 1e30f)) return GOOSE_EINVAL;
+    {
+        int impl = c->attn_impl;
+        if (impl == GOOSE_ATTN_AUTO) impl = goose::auto_attn_impl(c, S, B, H);
+        if (impl == GOOSE_ATTN_UMMA && S > 0) {
+            cudaError_t ea = goose::launch_tree_attn_umma(c, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_cache,
+                                                          (const __nv_bfloat16*)v_cache, kv_rows, row_off, ctx_len, parent,
+                                                          n_nodes, S, B, H, Hkv, scale, (__nv_bfloat16*)out, lse,
+                                                          static_cast<cudaStream_t>(stream), &merge_plan);
+            if (ea != cudaSuccess) return cuda_fail(ea);
+        } else {
+            rc = goose_tree_attn_gqa(c, q, k_cache, v_cache, kv_rows, row_off, ctx_len, parent, n_nodes, S, B, H, Hkv, D, scale,
+                                     out, lse, stream);
+            if (rc) return rc;
+        }
+    }
     // the logits are an input of the step: complete before the attention kernels above started, which do not touch
     // them -- so the top-k kernel may read them while the attention merge is still running.  With a harvest it also
     // returns every row's log-sum-exp (one pass over the logits serves the walk and the table).
@@ -338,7 +357,7 @@ int enqueue_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int6
     cudaError_t e = goose::launch_accept_compact(c, (__nv_bfloat16*)k_cache, (__nv_bfloat16*)v_cache, row_off, ctx_len,
                                                  draft_tok, parent, n_nodes, argmax, S, B, Hkv, kv_rows, path, accept_len, bonus,
                                                  new_ctx_len, static_cast<cudaStream_t>(stream), table_rows, k, topk_ids,
-                                                 topk_vals, row_lse, harvest ? adj_ids : nullptr, adj_scores);
+                                                 topk_vals, row_lse, harvest ? adj_ids : nullptr, adj_scores, &merge_plan);
     if (e != cudaSuccess) return cuda_fail(e);
     return GOOSE_OK;
 }

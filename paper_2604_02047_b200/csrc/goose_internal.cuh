@@ -125,7 +125,8 @@ cudaError_t launch_accept_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16
                                   int32_t* accept_len, int32_t* bonus, int32_t* new_ctx, cudaStream_t st,
                                   int table_rows = 0, int k = 0, const int32_t* topk_ids = nullptr,
                                   const float* topk_vals = nullptr, const float* row_lse = nullptr,
-                                  int32_t* adj_ids = nullptr, float* adj_scores = nullptr);
+                                  int32_t* adj_ids = nullptr, float* adj_scores = nullptr,
+                                  const struct CombinePlan* merge = nullptr);
 cudaError_t launch_tree_attn_mma(goose_ctx* c, const __nv_bfloat16* q, const __nv_bfloat16* kc,
                                  const __nv_bfloat16* vc, int64_t kv_rows, const int64_t* row_off, const int32_t* ctx_len,
                                  const int32_t* parent, const int32_t* n_nodes, int S, int B, int H, int Hkv, float scale,
@@ -133,7 +134,8 @@ cudaError_t launch_tree_attn_mma(goose_ctx* c, const __nv_bfloat16* q, const __n
 cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __nv_bfloat16* kc,
                                   const __nv_bfloat16* vc, int64_t kv_rows, const int64_t* row_off,
                                   const int32_t* ctx_len, const int32_t* parent, const int32_t* n_nodes, int S, int B, int H,
-                                  int Hkv, float scale, __nv_bfloat16* out, float* lse, cudaStream_t st);
+                                  int Hkv, float scale, __nv_bfloat16* out, float* lse, cudaStream_t st,
+                                  struct CombinePlan* defer_merge = nullptr);
 
 cudaError_t launch_bounded_wait_selftest(goose_ctx* c, long long limit_cycles, int32_t* result, cudaStream_t st);
 

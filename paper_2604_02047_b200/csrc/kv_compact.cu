@@ -7,6 +7,7 @@
 // stores; a batch's destinations are below every later source), which keeps 8 loads in flight per
 // thread without any barrier.
 #include "goose_internal.cuh"
+#include "tree_attn_combine.cuh"
 
 namespace goose {
 
@@ -101,8 +102,9 @@ cudaError_t launch_kv_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc
 // With a harvest (adj_ids != NULL) the launch carries a third block role, blockIdx.y == 2: one warp per logits row of the
 // sequence writes that row's top-k ids and softmax scores to adjacency-table row draft_tok[row] unless a later row of the
 // call carries the same token -- the rule of harvest_scatter_kernel, decided here before the wait (tokens are inputs).
-template <bool kCounts>
-__global__ void __launch_bounds__(kCompactThreads)
+// kMerge: 0 = no merge role, 1 = merge of multi-head attention, 2 = of grouped-query attention (256 threads then)
+template <bool kCounts, int kMerge>
+__global__ void __launch_bounds__(kMerge ? kCombineThreads : kCompactThreads)
 accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __restrict__ row_off,
                       const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ draft_tok,
                       const int32_t* __restrict__ parent, const int32_t* __restrict__ n_nodes,
@@ -112,8 +114,20 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
                       int32_t* __restrict__ status,
                       int rows_total, int table_rows, int k, const int32_t* __restrict__ topk_ids,
                       const float* __restrict__ topk_vals, const float* __restrict__ row_lse,
-                      int32_t* __restrict__ adj_ids, float* __restrict__ adj_scores) {
+                      int32_t* __restrict__ adj_ids, float* __restrict__ adj_scores,
+                      int base_roles, int merge_row_groups, const CombineArgs ca) {
     if (!kCounts) n_nodes = nullptr;
+    constexpr int kT = kMerge ? kCombineThreads : kCompactThreads;   // threads of this launch
+    if (kMerge && (int)blockIdx.y >= base_roles) {
+        // ---- merge role: 32 rows of one head of the attention work list (the partials of the step's main kernel)
+        if ((int)blockIdx.x >= merge_row_groups) {      // the grid is as wide as its widest role
+            pdl_wait();
+            pdl_trigger();
+            return;
+        }
+        combine_heads<kMerge == 2, kCounts>(ca, blockIdx.x, (int)blockIdx.y - base_roles, blockIdx.z);
+        return;
+    }
 
     __shared__ int s_path[kMaxB];
     __shared__ int s_len;
@@ -125,7 +139,7 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
     if (blockIdx.y == 2) {
         // ---- harvest scatter role
         const int lane = threadIdx.x & 31;
-        const int i = blockIdx.x * (kCompactThreads / 32) + (threadIdx.x >> 5);   // node of sequence s
+        const int i = blockIdx.x * (kT / 32) + (threadIdx.x >> 5);   // node of sequence s
         const size_t r = (size_t)s * B + i;
         int tok = -1;
         bool write = false;
@@ -149,13 +163,13 @@ accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __res
         }
         return;
     }
-    if ((int)blockIdx.x * kCompactThreads >= row_vec) {   // the grid is as wide as its widest role: nothing to copy here
+    if ((int)blockIdx.x * kT >= row_vec) {   // the grid is as wide as its widest role: nothing to copy here
         pdl_wait();
         pdl_trigger();
         return;
     }
     const int which = blockIdx.y;                        // 0 = K, 1 = V
-    const int col = blockIdx.x * kCompactThreads + threadIdx.x;
+    const int col = blockIdx.x * kT + threadIdx.x;
     const bool publisher = blockIdx.x == 0 && which == 0;
     // rows this sequence owns must lie inside the cache: never form an address from unchecked device data
     const int ctx0 = ctx_len[s];
@@ -249,19 +263,34 @@ cudaError_t launch_accept_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16
                                   const int32_t* n_nodes, const int32_t* argmax, int S, int B, int H, int64_t kv_rows, int32_t* path,
                                   int32_t* accept_len, int32_t* bonus, int32_t* new_ctx, cudaStream_t st,
                                   int table_rows, int k, const int32_t* topk_ids, const float* topk_vals,
-                                  const float* row_lse, int32_t* adj_ids, float* adj_scores) {
+                                  const float* row_lse, int32_t* adj_ids, float* adj_scores, const CombinePlan* merge) {
     if (S == 0) return cudaSuccess;
+    const bool with_merge = merge && merge->valid;     // the attention merge of this step rides in this launch
+    const int threads = with_merge ? kCombineThreads : kCompactThreads;
     int row_vec = H * kHeadDim * 2 / 16;
-    int gx = (row_vec + kCompactThreads - 1) / kCompactThreads;
+    int gx = (row_vec + threads - 1) / threads;
     const bool scatter = adj_ids != nullptr;
     if (scatter) {
-        const int sx = (B + kCompactThreads / 32 - 1) / (kCompactThreads / 32);   // one warp per logits row
+        const int sx = (B + threads / 32 - 1) / (threads / 32);   // one warp per logits row
         if (sx > gx) gx = sx;
     }
-    dim3 grid(gx, scatter ? 3 : 2, S);
-    cudaError_t e = launch_pdl(n_nodes ? accept_compact_kernel<true> : accept_compact_kernel<false>, grid, dim3(kCompactThreads), 0, st, kc, vc, row_off, ctx_len,
+    const int base_roles = scatter ? 3 : 2;
+    CombineArgs ca{};
+    int merge_rg = 0, roles = base_roles;
+    if (with_merge) {
+        ca = merge->args; merge_rg = merge->row_groups; roles += ca.Hw;
+        if (merge_rg > gx) gx = merge_rg;
+    }
+    dim3 grid(gx, roles, S);
+    const bool counts = n_nodes != nullptr;
+    const int mode = !with_merge ? 0 : (merge->grouped ? 2 : 1);
+    auto kernel = mode == 0 ? (counts ? accept_compact_kernel<true, 0> : accept_compact_kernel<false, 0>)
+                : mode == 1 ? (counts ? accept_compact_kernel<true, 1> : accept_compact_kernel<false, 1>)
+                            : (counts ? accept_compact_kernel<true, 2> : accept_compact_kernel<false, 2>);
+    cudaError_t e = launch_pdl(kernel, grid, dim3(threads), 0, st, kc, vc, row_off, ctx_len,
                                draft_tok, parent, n_nodes, argmax, B, row_vec, kv_rows, path, accept_len, bonus, new_ctx, c->status,
-                               S * B, table_rows, k, topk_ids, topk_vals, row_lse, adj_ids, adj_scores);
+                               S * B, table_rows, k, topk_ids, topk_vals, row_lse, adj_ids, adj_scores,
+                               base_roles, merge_rg, ca);
     c->launches++;
     return e;
 }

@@ -30,12 +30,12 @@
 #include <cuda_fp16.h>
 
 #include "goose_internal.cuh"
+#include "tree_attn_combine.cuh"
 
 namespace goose {
 
 namespace {
 
-constexpr int kTile = 128;                      // keys per tile
 constexpr int kStages = 5;                      // ring of K/V stages (P lives in tensor memory, not here)
 constexpr int kStageBytes = kTile * kHeadDim * 2;   // 32 KB: one K or one V tile
 constexpr int kHalfBytes = kTile * 128;         // 16 KB: 128 rows x 64 bf16 (one swizzle-atom column)
@@ -46,14 +46,7 @@ constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;       // rescale O only when the running max grew by > 2^8
-constexpr int kCombineThreads = 256;
-constexpr int kCombineRound = 4;                 // partials merged per load round of the combine kernel
-// split-KV partial of this kernel: normalised O/l as fp16, uint4 [16 column groups of 8][128 rows] (32 KB, a warp's
-// stores and the combine kernel's loads are contiguous), then m[128], l[128] as fp32
-constexpr int kPartHalfWords = 16 * 128 * 4;     // 32-bit words of the fp16 block
-constexpr int kUmmaPartFloats = kPartHalfWords + 2 * kMaxB;
 constexpr long long kWaitCycles = 2000000000ll;  // bound of every wait: about one second of SM clock
 
 struct Header {                                  // lives at the start of dynamic shared memory
@@ -187,16 +180,6 @@ __device__ __forceinline__ void umma_commit(unsigned long long* bar) {
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-__device__ __forceinline__ float ex2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
 // barrier of the 128 softmax threads; `n` counts its uses (every thread calls it the same number of times)
 __device__ __forceinline__ bool group_sync(Header* hd, uint32_t& n, int32_t* status) {
     mbar_arrive(&hd->group_bar);
@@ -204,69 +187,6 @@ __device__ __forceinline__ bool group_sync(Header* hd, uint32_t& n, int32_t* sta
     ++n;
     return ok;
 }
-
-// ---------------------------------------------------------------- work partition (same code in every role)
-struct Work {
-    const int32_t* ctx_len;
-    const int32_t* n_nodes;   // per-sequence node counts, or NULL (every tree has B nodes)
-    int S, H, B, G;           // H = heads of the work list = M tiles x key/value heads (M-tile-major)
-    long long total;          // all items
-    bool small;               // total * (G + 1) fits 31 bits: 32-bit arithmetic (64-bit division is slow on the GPU)
-    // ctx_len comes from device memory: a negative value is treated as 0 (the tree rows alone).  A sequence's keys are
-    // its prefix and the nodes its tree really has; a sequence without nodes (it has left the batch) has no items.
-    __device__ __forceinline__ int tiles(int s) const {
-        if (!n_nodes) return (max(ctx_len[s], 0) + B + kTile - 1) / kTile;
-        const int nn = nodes_of(n_nodes, s, B);
-        return nn == 0 ? 0 : (max(ctx_len[s], 0) + nn + kTile - 1) / kTile;
-    }
-    __device__ __forceinline__ void init() {
-        long long tot = 0;
-        for (int s = 0; s < S; ++s) tot += (long long)H * tiles(s);
-        total = tot;
-        small = tot * (G + 1) < 0x7FFFFFFFll;
-    }
-    __device__ __forceinline__ long long cta_start(int c) const {
-        if (small) return ((uint32_t)total * (uint32_t)c) / (uint32_t)G;
-        return total * c / G;
-    }
-    __device__ __forceinline__ int cta_of(long long w) const {
-        int c = small ? (int)(((uint32_t)w * (uint32_t)G) / (uint32_t)total) : (int)(w * G / total);
-        if (c >= G) c = G - 1;
-        while (c + 1 < G && cta_start(c + 1) <= w) ++c;
-        while (c > 0 && cta_start(c) > w) --c;
-        return c;
-    }
-};
-
-struct Cursor {               // walks items in order
-    long long w;              // item index
-    int s, h, t, T;
-    __device__ __forceinline__ void seek(const Work& wk, long long w0) {
-        long long off = 0;
-        int ss = 0;
-        int TT = wk.tiles(0);
-        while (ss + 1 < wk.S && off + (long long)wk.H * TT <= w0) {
-            off += (long long)wk.H * TT;
-            ++ss;
-            TT = wk.tiles(ss);
-        }
-        s = ss; T = TT; w = w0;
-        const long long rem = w0 - off;
-        h = wk.small ? (int)((uint32_t)rem / (uint32_t)TT) : (int)(rem / TT);
-        t = (int)(rem - (long long)h * TT);
-    }
-    __device__ __forceinline__ void next(const Work& wk) {
-        ++w; ++t;
-        if (t == T) {
-            t = 0; ++h;
-            if (h == wk.H) {                              // next sequence that has any items
-                h = 0; ++s;
-                if (!wk.n_nodes) { if (s < wk.S) T = wk.tiles(s); }
-                else while (s < wk.S && (T = wk.tiles(s)) == 0) ++s;
-            }
-        }
-    }
-};
 
 // ---------------------------------------------------------------- the kernel
 // kGrouped = false is multi-head attention: one query head per key/value head and one M tile per sequence are
@@ -700,107 +620,6 @@ tree_attn_umma_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     }
 }
 
-// ---------------------------------------------------------------- combine of the split-KV partials
-// Grid (row groups of 32, M tiles x key/value heads, S), 256 threads.  A head of the work list that one CTA of the
-// main kernel covered entirely was written directly and is skipped; any other is the merge of its CTAs' partials:
-//   M = max m_p,  L = sum l_p 2^(m_p - M),  out = sum_p 2^(m_p - M) O_p / L.
-// Lane <-> row (coalesced float4 loads of the transposed partial layout), warp <-> 16 output columns.
-template <bool kGrouped, bool kCounts>
-__global__ void __launch_bounds__(kCombineThreads)
-tree_attn_combine_kernel(const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ n_nodes, int S, int B, int H,
-                         int Hkv_arg, int g_arg, int nb_arg, int G,
-                         const float* __restrict__ partials, __nv_bfloat16* __restrict__ out,
-                         float* __restrict__ lse) {
-    if (!kCounts) n_nodes = nullptr;
-
-    const int Hkv = kGrouped ? Hkv_arg : H, g = kGrouped ? g_arg : 1, nb = kGrouped ? nb_arg : B;
-    const int rg = blockIdx.x, h = blockIdx.y, s = blockIdx.z;   // h = head of the work list (M tile, KV head)
-    const int Hw = gridDim.y;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // The partition arithmetic needs only ctx_len[], which is final before this kernel's CTAs can start: the main
-    // kernel triggers its dependents after its own pdl_wait(), i.e. after whatever produced ctx_len[] completed.
-    // So all of it runs before the wait, and the partial loads are issued the moment the main grid is done.
-    Work wk;
-    wk.ctx_len = ctx_len; wk.n_nodes = n_nodes; wk.S = S; wk.H = Hw; wk.B = B; wk.G = G;
-    wk.init();
-    long long off = 0;
-    for (int ss = 0; ss < s; ++ss) off += (long long)Hw * wk.tiles(ss);
-    const int T = wk.tiles(s);                             // 0: the sequence has no nodes, hence no items and no output
-    const long long head_first = off + (long long)h * T;
-    const bool any = !kCounts || T > 0;                    // (without counts every sequence has tiles)
-    const int c_lo = any ? wk.cta_of(head_first) : 0, c_hi = any ? wk.cta_of(head_first + T - 1) : 0;
-    const bool whole = c_lo == c_hi;                       // written directly by the main kernel (or nothing to write)
-    const int row = rg * 32 + lane;                        // row of the M tile = (node of the tile, head of the group)
-    const int mt = kGrouped ? h / Hkv : 0, hk = h - mt * Hkv;
-    const int i_local = kGrouped ? row / g : row, node = mt * nb + i_local;
-    const int hq = hk * g + (row - i_local * g);
-    const bool row_valid = i_local < nb && node < nodes_of(n_nodes, s, B);
-    // CTA c's partial for this head sits in slot 2c, or 2c+1 when its segment starts at the head's first tile,
-    // which only the first CTA can do.  With fewer items than CTAs some CTAs in [c_lo, c_hi] are empty.
-    const int flag_lo = wk.cta_start(c_lo) <= head_first ? 1 : 0;
-    const bool sparse = wk.total < G;
-    // every CTA waits, also those with nothing to do: the next kernel in the stream relies on "this grid is
-    // complete" implying "the main grid is complete"
-    pdl_wait();                                            // the main kernel's partials are complete and visible
-    pdl_trigger();
-    if (whole || !row_valid) return;
-    float M_run = -INFINITY, L_run = 0.f;
-    float acc[16];                                         // warp w owns columns 16w .. 16w+15 (column groups 2w, 2w+1)
-#pragma unroll
-    for (int u = 0; u < 16; ++u) acc[u] = 0.f;
-
-    // kCombineRound parts per round: their (m, l) and their two 16-byte pieces of O/l are loaded together
-    // (16 independent loads in flight per thread); a running (M, L) with rescaling merges the rounds
-    for (int cb = c_lo; cb <= c_hi; cb += kCombineRound) {
-        float mp[kCombineRound], lp[kCombineRound];
-        uint4 x[kCombineRound][2];
-#pragma unroll
-        for (int q = 0; q < kCombineRound; ++q) {
-            const int c = cb + q;
-            bool use = c <= c_hi;
-            if (use && sparse) use = wk.cta_start(c + 1) > wk.cta_start(c);
-            const int sl = use ? 2 * c + (c == c_lo ? flag_lo : 0) : 0;
-            const float* pp = partials + (size_t)sl * kUmmaPartFloats;
-            mp[q] = use ? __ldcg(pp + kPartHalfWords + row) : -INFINITY;
-            lp[q] = use ? __ldcg(pp + kPartHalfWords + kMaxB + row) : 0.f;
-            const uint4* p4 = reinterpret_cast<const uint4*>(pp) + row;
-#pragma unroll
-            for (int u = 0; u < 2; ++u)
-                x[q][u] = use ? __ldcg(p4 + (2 * warp + u) * 128) : make_uint4(0u, 0u, 0u, 0u);
-        }
-        float M_new = M_run;
-#pragma unroll
-        for (int q = 0; q < kCombineRound; ++q) M_new = fmaxf(M_new, mp[q]);
-        const float a_old = (M_run == -INFINITY) ? 0.f : ex2(M_run - M_new);
-        L_run *= a_old;
-#pragma unroll
-        for (int u = 0; u < 16; ++u) acc[u] *= a_old;
-#pragma unroll
-        for (int q = 0; q < kCombineRound; ++q) {
-            const float w = ((mp[q] == -INFINITY) ? 0.f : ex2(mp[q] - M_new)) * lp[q];   // un-normalise: O_p = x_p * l_p
-            L_run += w;
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-                const uint32_t hw[4] = {x[q][u].x, x[q][u].y, x[q][u].z, x[q][u].w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&hw[e]));
-                    acc[8 * u + 2 * e] += w * f.x;
-                    acc[8 * u + 2 * e + 1] += w * f.y;
-                }
-            }
-        }
-        M_run = M_new;
-    }
-    const float inv = 1.f / L_run;
-    uint4* dst = reinterpret_cast<uint4*>(out + (((size_t)s * B + node) * H + hq) * kHeadDim + 16 * warp);
-#pragma unroll
-    for (int u = 0; u < 2; ++u)
-        dst[u] = make_uint4(pack_bf16x2(acc[8 * u] * inv, acc[8 * u + 1] * inv), pack_bf16x2(acc[8 * u + 2] * inv, acc[8 * u + 3] * inv),
-                            pack_bf16x2(acc[8 * u + 4] * inv, acc[8 * u + 5] * inv), pack_bf16x2(acc[8 * u + 6] * inv, acc[8 * u + 7] * inv));
-    if (lse && warp == 0) lse[((size_t)s * B + node) * H + hq] = (M_run + log2f(L_run)) * kLn2;
-}
-
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -890,7 +709,9 @@ int auto_attn_impl(const goose_ctx* c, int S, int B, int H) {
 cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __nv_bfloat16* kc,
                                   const __nv_bfloat16* vc, int64_t kv_rows, const int64_t* row_off,
                                   const int32_t* ctx_len, const int32_t* parent, const int32_t* n_nodes, int S, int B, int H,
-                                  int Hkv, float scale, __nv_bfloat16* out, float* lse, cudaStream_t st) {
+                                  int Hkv, float scale, __nv_bfloat16* out, float* lse, cudaStream_t st,
+                                  CombinePlan* defer_merge) {
+    if (defer_merge) defer_merge->valid = false;
     if (!c->encode_tiled) return cudaErrorNotSupported;
     if (S == 0) return cudaSuccess;
     const int g = H / Hkv;                              // query heads per key/value head (validated by the caller)
@@ -907,17 +728,23 @@ cudaError_t launch_tree_attn_umma(goose_ctx* c, const __nv_bfloat16* q, const __
     const bool counts = n_nodes != nullptr;
     auto main_kernel = grouped ? (counts ? tree_attn_umma_kernel<true, true> : tree_attn_umma_kernel<true, false>)
                                : (counts ? tree_attn_umma_kernel<false, true> : tree_attn_umma_kernel<false, false>);
-    auto merge_kernel = grouped ? (counts ? tree_attn_combine_kernel<true, true> : tree_attn_combine_kernel<true, false>)
-                                : (counts ? tree_attn_combine_kernel<false, true> : tree_attn_combine_kernel<false, false>);
     cudaError_t e = launch_pdl(main_kernel, dim3(grid),
                                dim3(kThreads), kUmmaSmem, st, mq, mk, mv, row_off, ctx_len, parent, n_nodes, S, B, H, Hkv, g, nb,
                                kv_rows, scale * kLog2e, c->partials, c->status, out, lse);
     c->launches++;
     if (e != cudaSuccess) return e;
-    dim3 cgrid((nb * g + 31) / 32, n_mt * Hkv, S);
-    const float* parts = c->partials;
-    e = launch_pdl(merge_kernel, cgrid,
-                   dim3(kCombineThreads), 0, st, ctx_len, n_nodes, S, B, H, Hkv, g, nb, grid, parts, out, lse);
+    CombineArgs ca;
+    ca.ctx_len = ctx_len; ca.n_nodes = n_nodes; ca.S = S; ca.B = B; ca.H = H; ca.Hkv = Hkv; ca.g = g; ca.nb = nb;
+    ca.G = grid; ca.Hw = n_mt * Hkv; ca.partials = c->partials; ca.out = out; ca.lse = lse;
+    const int row_groups = (nb * g + 31) / 32;
+    if (defer_merge) {                                  // the caller runs the merge as a role of a later launch
+        defer_merge->args = ca; defer_merge->row_groups = row_groups; defer_merge->grouped = grouped;
+        defer_merge->valid = true;
+        return cudaSuccess;
+    }
+    auto merge_kernel = grouped ? (counts ? tree_attn_combine_kernel<true, true> : tree_attn_combine_kernel<true, false>)
+                                : (counts ? tree_attn_combine_kernel<false, true> : tree_attn_combine_kernel<false, false>);
+    e = launch_pdl(merge_kernel, dim3(row_groups, ca.Hw, S), dim3(kCombineThreads), 0, st, ca);
     c->launches++;
     return e;
 }

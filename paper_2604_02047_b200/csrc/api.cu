@@ -340,8 +340,8 @@ int enqueue_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int6
             if (rc) return rc;
         }
     }
-    // the logits are an input of the step: complete before the attention kernels above started, which do not touch
-    // them -- so the top-k kernel may read them while the attention merge is still running.  With a harvest it also
+    // the logits are an input of the step: complete before the attention kernel above started, which does not touch
+    // them -- so the top-k kernel may read them while that kernel is still running.  With a harvest it also
     // returns every row's log-sum-exp (one pass over the logits serves the walk and the table).
     if (S > 0) {
         // (with logits_ready the kernel cannot start before the event, so reading ahead of its own wait stays safe)

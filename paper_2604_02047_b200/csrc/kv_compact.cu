@@ -102,7 +102,11 @@ cudaError_t launch_kv_compact(goose_ctx* c, __nv_bfloat16* kc, __nv_bfloat16* vc
 // With a harvest (adj_ids != NULL) the launch carries a third block role, blockIdx.y == 2: one warp per logits row of the
 // sequence writes that row's top-k ids and softmax scores to adjacency-table row draft_tok[row] unless a later row of the
 // call carries the same token -- the rule of harvest_scatter_kernel, decided here before the wait (tokens are inputs).
-// kMerge: 0 = no merge role, 1 = merge of multi-head attention, 2 = of grouped-query attention (256 threads then)
+// With the tensor-core attention kernel the launch also carries the merge of that kernel's split heads (kMerge: 0 = no
+// merge role, 1 = multi-head, 2 = grouped-query attention; 256 threads per CTA then): blockIdx.y >= base_roles is head
+// blockIdx.y - base_roles of the attention work list, blockIdx.x its group of 32 rows.  The merge needs the main kernel
+// to be complete, which this launch's dependency wait implies (every CTA of the top-k kernel in between has waited for
+// it), and nothing of the walk: it simply runs beside it instead of standing between the attention kernel and the top-k.
 template <bool kCounts, int kMerge>
 __global__ void __launch_bounds__(kMerge ? kCombineThreads : kCompactThreads)
 accept_compact_kernel(__nv_bfloat16* kc, __nv_bfloat16* vc, const int64_t* __restrict__ row_off,

@@ -106,7 +106,7 @@ node_topk_kernel(const __nv_bfloat16* __restrict__ logits, long long items_all, 
     if (tid < 32) s_list[tid] = 0;
     __syncthreads();
     // inputs_ready: the caller guarantees that the logits were complete before the preceding kernel in the stream
-    // started (the whole-step call: that kernel is the attention merge, which neither reads nor writes them).  The
+    // started (the whole-step call: that kernel is the attention kernel, which neither reads nor writes them).  The
     // CTA then streams and selects at once and only waits for the preceding kernel before its first write to global
     // memory (outputs, cross-CTA scratch); otherwise it waits here, before its first read.
     bool waited = inputs_ready == 0;

@@ -137,6 +137,9 @@ int goose_destroy(goose_ctx* c) {
     if (c->side) cudaStreamDestroy(c->side);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_logits) cudaEventDestroy(c->ev_logits);
+    if (c->side_down) cudaStreamDestroy(c->side_down);
+    if (c->ev_attn) cudaEventDestroy(c->ev_attn);
+    if (c->ev_out) cudaEventDestroy(c->ev_out);
     delete c;
     return GOOSE_OK;
 }
@@ -277,7 +280,7 @@ int enqueue_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int6
                  void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
                  int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
                  float* row_lse, int table_rows, int32_t* adj_ids, float* adj_scores, void* stream,
-                 cudaEvent_t logits_ready);
+                 cudaEvent_t logits_ready, cudaEvent_t attn_done = nullptr);
 }  // namespace
 
 extern "C" {
@@ -304,7 +307,7 @@ int enqueue_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int6
                  void* out, float* lse, int32_t* argmax, int32_t* topk_ids, float* topk_vals,
                  int32_t* path, int32_t* accept_len, int32_t* bonus, int32_t* new_ctx_len,
                  float* row_lse, int table_rows, int32_t* adj_ids, float* adj_scores, void* stream,
-                 cudaEvent_t logits_ready) {
+                 cudaEvent_t logits_ready, cudaEvent_t attn_done) {
     // validate everything before enqueueing anything
     const bool harvest = row_lse || adj_ids || adj_scores;
     if (harvest && (!row_lse || !adj_ids || !adj_scores || !topk_vals || table_rows < 1)) return GOOSE_EINVAL;
@@ -328,7 +331,9 @@ int enqueue_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int6
     {
         int impl = c->attn_impl;
         if (impl == GOOSE_ATTN_AUTO) impl = goose::auto_attn_impl(c, S, B, H);
-        if (impl == GOOSE_ATTN_UMMA && S > 0) {
+        // attn_done (the host-buffer call): out[] must be complete as early as possible, so that it can travel to the
+        // host while the logits are still on their way up -- the attention then keeps the merge as its own kernel
+        if (impl == GOOSE_ATTN_UMMA && S > 0 && !attn_done) {
             cudaError_t ea = goose::launch_tree_attn_umma(c, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k_cache,
                                                           (const __nv_bfloat16*)v_cache, kv_rows, row_off, ctx_len, parent,
                                                           n_nodes, S, B, H, Hkv, scale, (__nv_bfloat16*)out, lse,
@@ -339,6 +344,7 @@ int enqueue_step(goose_ctx* c, const void* q, void* k_cache, void* v_cache, int6
                                      out, lse, stream);
             if (rc) return rc;
         }
+        if (attn_done) GOOSE_CUDA(cudaEventRecord(attn_done, static_cast<cudaStream_t>(stream)));
     }
     // the logits are an input of the step: complete before the attention kernel above started, which does not touch
     // them -- so the top-k kernel may read them while that kernel is still running.  With a harvest it also
@@ -436,6 +442,9 @@ int goose_verify_step_host_gqa(goose_ctx* c, void* k_cache, void* v_cache, int64
         GOOSE_CUDA(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking));
         GOOSE_CUDA(cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming));
         GOOSE_CUDA(cudaEventCreateWithFlags(&c->ev_logits, cudaEventDisableTiming));
+        GOOSE_CUDA(cudaStreamCreateWithFlags(&c->side_down, cudaStreamNonBlocking));
+        GOOSE_CUDA(cudaEventCreateWithFlags(&c->ev_attn, cudaEventDisableTiming));
+        GOOSE_CUDA(cudaEventCreateWithFlags(&c->ev_out, cudaEventDisableTiming));
     }
     const size_t in_bytes = o_nn + (size_t)S * 4 - o_rowoff;       // row_off | ctx_len | parent | draft_tok | n_nodes (padded as above)
     const size_t out_bytes = o_newctx + (size_t)S * 4 - o_argmax;  // argmax | ids | vals | path | accept_len | bonus | new_ctx
@@ -480,13 +489,18 @@ int goose_verify_step_host_gqa(goose_ctx* c, void* k_cache, void* v_cache, int64
                       d + o_logits, V, S, B, H, Hkv, D, V, k, scale, d + o_out, nullptr, (int32_t*)(d + o_argmax),
                       (int32_t*)(d + o_ids), (float*)(d + o_vals), (int32_t*)(d + o_path),
                       (int32_t*)(d + o_alen), (int32_t*)(d + o_bonus), (int32_t*)(d + o_newctx), nullptr, 0, nullptr, nullptr,
-                      stream, c->ev_logits);
+                      stream, c->ev_logits, c->ev_attn);
     if (rc) {
         cudaStreamSynchronize(c->side);                  // nothing of this call may stay in flight behind an error
         return rc;
     }
-    GOOSE_CUDA(cudaMemcpyAsync(h_out, d + o_out, n_q, cudaMemcpyDeviceToHost, st));
+    // the attention output goes down on its own stream as soon as the attention is done: the link carries it while the
+    // logits are still going up the other way
+    GOOSE_CUDA(cudaStreamWaitEvent(c->side_down, c->ev_attn, 0));
+    GOOSE_CUDA(cudaMemcpyAsync(h_out, d + o_out, n_q, cudaMemcpyDeviceToHost, c->side_down));
+    GOOSE_CUDA(cudaEventRecord(c->ev_out, c->side_down));
     GOOSE_CUDA(cudaMemcpyAsync(pin_out, d + o_argmax, out_bytes, cudaMemcpyDeviceToHost, st));   // the small results: one copy
+    GOOSE_CUDA(cudaStreamWaitEvent(st, c->ev_out, 0));
     GOOSE_CUDA(cudaStreamSynchronize(st));
     memcpy(h_argmax, pin_out + (o_argmax - o_argmax), rows * 4);
     memcpy(h_topk_ids, pin_out + (o_ids - o_argmax), rows * k * 4);

@@ -43,7 +43,8 @@ struct goose_ctx {
     void* pin;                // pinned host block: the small input arrays go up, the small results come down, in one copy each
     size_t pin_bytes;
     cudaStream_t side;        // the logits are uploaded here, next to the attention kernels
-    cudaEvent_t ev_fork, ev_logits;
+    cudaStream_t side_down;   // the attention output goes down here while the logits are still going up
+    cudaEvent_t ev_fork, ev_logits, ev_attn, ev_out;
     long long launches;
     void* encode_tiled;       // cuTensorMapEncodeTiled entry point (driver), resolved at create
 };

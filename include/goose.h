@@ -201,8 +201,10 @@ int goose_kv_compact(goose_ctx* ctx, void* k_cache, void* v_cache, int64_t kv_ro
                      int32_t* new_ctx_len, void* stream);
 
 /* The whole step on one stream, in data-flow order: tree attention, node top-k (rows = S*B),
- * acceptance walk, KV compaction (the last two share one launch).  Arguments and results as in the
- * four calls above (new_ctx_len must not overlap ctx_len).  q, the caches' tree rows, parent, draft_tok,
+ * acceptance walk, KV compaction (the last two share one launch, which with the tensor-core attention
+ * kernel also finishes the attention: the merge of its split heads runs there, beside the walk).  All
+ * results, out and lse included, are complete in stream order when the call's last kernel is.  Arguments
+ * and results as in the four calls above (new_ctx_len must not overlap ctx_len).  q, the caches' tree rows, parent, draft_tok,
  * logits, ctx_len and row_off are INPUTS of the step: they must be complete in stream order before the
  * call and nothing else may write them until the step is done; some kernels of the step read them
  * ahead of their stream-order dependency on the step's earlier kernels.                              */
@@ -251,8 +253,9 @@ int goose_verify_step_harvest(goose_ctx* ctx, const void* q, void* k_cache, void
  *        h_path [S][B]; h_accept_len, h_bonus, h_new_ctx_len [S]
  * Copies in, runs goose_verify_step, copies out, and synchronises `stream` before returning.
  * The logits (most of the bytes, needed by the top-k only) are uploaded on a stream of the context's own while the
- * attention kernels run; the small arrays travel through one pinned block of the context, one copy each way.
- * Device and pinned staging buffers, that stream and its events are created inside the context on first use and
+ * attention kernels run, and h_out is copied down on another one as soon as the attention is done; the small arrays
+ * travel through one pinned block of the context, one copy each way.
+ * Device and pinned staging buffers, those streams and their events are created inside the context on first use and
  * grow on demand; calls on one context must not overlap.                                                     */
 int goose_verify_step_host(goose_ctx* ctx, void* k_cache, void* v_cache, int64_t kv_rows,
                            const void* h_q, const void* h_k_new, const void* h_v_new,
